@@ -1,0 +1,327 @@
+"""Pins for the CPU oracle: each routine is checked against something other than
+itself -- a hand-worked example, closed forms, numpy library routines for the
+no-decay case, a literal brute-force loop, finite differences, and the other
+form of the same function.  No GPU involved."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import la_oracle as orc
+from paper_2307_14995_b200 import inputs
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def rand_inputs(B, H, N, d, e, seed=0, dtype=torch.float32):
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, e, dtype=dtype, seed=seed)
+    return q, k, v, do
+
+
+def brute_forward(q, k, v, lam):
+    """The defining sum o_t = sum_{s<=t} lambda^(t-s) (q_t . k_s) v_s as literal Python loops."""
+    q, k, v = (np.asarray(x, dtype=np.float64) for x in (q, k, v))
+    B, H, N, d = q.shape
+    e = v.shape[-1]
+    o = np.zeros((B, H, N, e))
+    for b in range(B):
+        for h in range(H):
+            for t in range(N):
+                for s in range(t + 1):
+                    dot = 0.0
+                    for i in range(d):
+                        dot += q[b, h, t, i] * k[b, h, s, i]
+                    w = float(lam[h]) ** (t - s)
+                    for j in range(e):
+                        o[b, h, t, j] += w * dot * v[b, h, s, j]
+    return o
+
+
+def relerr(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    rms = np.sqrt(np.mean(b * b)) + 1e-300
+    return np.max(np.abs(a - b)) / rms
+
+
+# --- hand-worked example ------------------------------------------------------
+def test_hand_worked_example():
+    g = json.load(open(os.path.join(HERE, "golden", "hand_example.json")))
+    sh = (1, 1, 3, 1)
+    q, k, v, do = (np.array(g[n], np.float32).reshape(sh) for n in ("q", "k", "v", "dO"))
+    lam = np.array([g["lambda"]])
+    o, kv = orc.fwd_rec(q, k, v, lam, want_state=True)
+    assert np.array_equal(o.ravel(), np.array(g["o"]))
+    assert kv.ravel()[0] == g["kv_out"]
+    assert np.array_equal(orc.fwd_quad(q, k, v, lam).ravel(), np.array(g["o"]))
+    for fn in (lambda: orc.bwd_rec(q, k, v, do, lam), lambda: orc.bwd_quad(q, k, v, do, lam)):
+        dq, dk, dv = fn()
+        assert np.array_equal(dq.ravel(), np.array(g["dq"]))
+        assert np.array_equal(dk.ravel(), np.array(g["dk"]))
+        assert np.array_equal(dv.ravel(), np.array(g["dv"]))
+    *_, gin = orc.bwd_rec(q, k, v, do, lam, want_state_grad=True)
+    assert gin.ravel()[0] == g["grad_kv_in"]
+    for kind in ("o", "dq", "dk", "dv"):
+        r = orc.rows(kind, q, k, v, do, lam, [0, 0, 0], [0, 1, 2])
+        assert np.array_equal(r.ravel(), np.array(g[kind]))
+
+
+# --- brute force on tiny inputs ----------------------------------------------
+@pytest.mark.parametrize("N,d,e", [(1, 1, 1), (5, 2, 3), (8, 3, 2)])
+def test_brute_force_tiny(N, d, e):
+    q, k, v, _ = rand_inputs(2, 2, N, d, e, seed=3)
+    lam = np.array([0.7, 1.0])
+    ref = brute_forward(q, k, v, lam)
+    assert relerr(orc.fwd_rec(q, k, v, lam), ref) < 1e-14
+    assert relerr(orc.fwd_quad(q, k, v, lam), ref) < 1e-14
+
+
+# --- closed forms ---------------------------------------------------------------
+@pytest.mark.parametrize("lam", [float(np.exp(-2.0)), 0.5, 1.0])
+def test_closed_form_geometric(lam):
+    """q_t = k_t = e_1, v_t = 1: o_t[j] = (1 - lam^(t+1)) / (1 - lam), or t+1 for lam = 1;
+    with dO = 1: dv_s[j] = (1 - lam^(N-s)) / (1 - lam)."""
+    N, d, e = 40, 3, 2
+    q = np.zeros((1, 1, N, d), np.float32)
+    q[..., 0] = 1.0
+    k = q.copy()
+    v = np.ones((1, 1, N, e), np.float32)
+    do = np.ones((1, 1, N, e), np.float32)
+    t = np.arange(N)
+    want_o = (t + 1.0) if lam == 1.0 else (1 - lam ** (t + 1)) / (1 - lam)
+    want_dv = (N - t).astype(float) if lam == 1.0 else (1 - lam ** (N - t)) / (1 - lam)
+    L = np.array([lam])
+    for o in (orc.fwd_rec(q, k, v, L), orc.fwd_quad(q, k, v, L)):
+        assert np.allclose(o[0, 0, :, 0], want_o, rtol=1e-13, atol=0)
+        assert np.allclose(o[0, 0, :, 1], want_o, rtol=1e-13, atol=0)
+    for dq, dk, dv in (orc.bwd_rec(q, k, v, do, L), orc.bwd_quad(q, k, v, do, L)):
+        assert np.allclose(dv[0, 0, :, 0], want_dv, rtol=1e-13, atol=0)
+        # dq_t = kv_t do_t = (sum_j kv[0,j]) e_1, and kv[0,j] = o_t[j]
+        assert np.allclose(dq[0, 0, :, 0], e * want_o, rtol=1e-13, atol=0)
+        assert np.all(dq[0, 0, :, 1:] == 0)
+        # dk_s = R_s v_s with R_s[0,j] = dv_s[j]
+        assert np.allclose(dk[0, 0, :, 0], e * want_dv, rtol=1e-13, atol=0)
+    if lam == float(np.exp(-2.0)):
+        long_q = np.zeros((1, 1, 400, 1), np.float32) + 1.0
+        o = orc.fwd_rec(long_q, long_q, long_q, L)
+        assert abs(o[0, 0, -1, 0] - 1.1565176427496657) < 1e-15
+
+
+def test_no_decay_is_prefix_sum():
+    """lambda = 1: O = tril(Q K^T) V, i.e. prefix sums of k_s v_s^T (numpy cumsum / tril)."""
+    q, k, v, do = rand_inputs(1, 2, 33, 4, 5, seed=5)
+    lam = np.array([1.0, 1.0])
+    qn, kn, vn, don = (x.double().numpy() for x in (q, k, v, do))
+    kv_prefix = np.cumsum(np.einsum("bhsi,bhsj->bhsij", kn, vn), axis=2)
+    want = np.einsum("bhti,bhtij->bhtj", qn, kv_prefix)
+    assert relerr(orc.fwd_rec(q, k, v, lam), want) < 1e-14
+    assert relerr(orc.fwd_quad(q, k, v, lam), want) < 1e-14
+    A = np.tril(np.einsum("bhti,bhsi->bhts", qn, kn))
+    dA = np.tril(np.einsum("bhtj,bhsj->bhts", don, vn))
+    want_g = (np.einsum("bhts,bhsi->bhti", dA, kn), np.einsum("bhts,bhti->bhsi", dA, qn),
+              np.einsum("bhts,bhtj->bhsj", A, don))
+    for got in (orc.bwd_rec(q, k, v, do, lam), orc.bwd_quad(q, k, v, do, lam)):
+        for g, w in zip(got, want_g):
+            assert relerr(g, w) < 1e-14
+
+
+def test_fast_decay_limit_is_diagonal():
+    """lambda -> 0: o_t = (q_t.k_t) v_t, dq_t = (do_t.v_t) k_t, dk_t = (do_t.v_t) q_t, dv_t = (q_t.k_t) do_t."""
+    q, k, v, do = rand_inputs(1, 1, 17, 4, 3, seed=7)
+    lam = np.array([1e-30])
+    qn, kn, vn, don = (x.double().numpy() for x in (q, k, v, do))
+    qk = np.sum(qn * kn, -1, keepdims=True)
+    dov = np.sum(don * vn, -1, keepdims=True)
+    for o in (orc.fwd_rec(q, k, v, lam), orc.fwd_quad(q, k, v, lam)):
+        assert np.all(np.isfinite(o)) and relerr(o, qk * vn) < 1e-14
+    for dq, dk, dv in (orc.bwd_rec(q, k, v, do, lam), orc.bwd_quad(q, k, v, do, lam)):
+        assert relerr(dq, dov * kn) < 1e-14
+        assert relerr(dk, dov * qn) < 1e-14
+        assert relerr(dv, qk * don) < 1e-14
+
+
+# --- the two forms against each other -----------------------------------------
+@pytest.mark.parametrize("shape", [(1, 2, 96, 8, 6), (2, 3, 257, 16, 16), (1, 1, 1, 4, 4)])
+def test_recurrence_equals_quadratic(shape):
+    B, H, N, d, e = shape
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=11)
+    lam = inputs.decay_rates(H, 0.5).double().numpy()
+    assert relerr(orc.fwd_rec(q, k, v, lam), orc.fwd_quad(q, k, v, lam)) < 1e-12
+    for a, b in zip(orc.bwd_rec(q, k, v, do, lam), orc.bwd_quad(q, k, v, do, lam)):
+        assert relerr(a, b) < 1e-12
+
+
+def test_recurrence_equals_quadratic_pr1_workload():
+    w = inputs.make_workload("pr1_ref")
+    lam = w["lam"].double().numpy()
+    assert np.allclose(lam, [1.0, np.exp(-2.0)], rtol=1e-7)
+    assert relerr(orc.fwd_rec(w["q"], w["k"], w["v"], lam), orc.fwd_quad(w["q"], w["k"], w["v"], lam)) < 1e-12
+    for a, b in zip(orc.bwd_rec(w["q"], w["k"], w["v"], w["do"], lam),
+                    orc.bwd_quad(w["q"], w["k"], w["v"], w["do"], lam)):
+        assert relerr(a, b) < 1e-12
+
+
+def test_sampled_rows_equal_full_forms():
+    B, H, N, d, e = 2, 2, 70, 8, 5
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=13)
+    lam = np.array([0.9, 0.3])
+    o = orc.fwd_rec(q, k, v, lam)
+    dq, dk, dv = orc.bwd_rec(q, k, v, do, lam)
+    bh = np.array([0, 1, 2, 3, 3, 0])
+    t = np.array([0, 69, 31, 32, 1, 68])
+    for kind, full in (("o", o), ("dq", dq), ("dk", dk), ("dv", dv)):
+        got = orc.rows(kind, q, k, v, do, lam, bh, t)
+        want = full.reshape(B * H, N, -1)[bh, t]
+        assert relerr(got, want) < 1e-12
+
+
+# --- gradients: finite differences, Euler identities, role swaps -------------------
+def test_finite_differences_including_state_gradients():
+    B, H, N, d, e = 1, 2, 12, 3, 4
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=17)
+    lam = np.array([0.8, 1.0])
+    rng = np.random.default_rng(0)
+    kv_in = rng.standard_normal((B, H, d, e))
+    gko = rng.standard_normal((B, H, d, e))
+    qn, kn, vn, don = (x.double().numpy().copy() for x in (q, k, v, do))
+
+    def loss(qq, kk, vv, s_in):
+        o, s_out = orc.fwd_rec(qq, kk, vv, lam, kv_in=s_in, want_state=True)
+        return float(np.sum(o * don) + np.sum(s_out * gko))
+
+    dq, dk, dv, gin = orc.bwd_rec(q, k, v, do, lam, kv_in=kv_in, grad_kv_out=gko, want_state_grad=True)
+    # inputs are fp32 containers: use perturbations that are exact in fp32 (power of two)
+    h = 2.0 ** -10
+    for name, arr, grad in (("q", qn, dq), ("k", kn, dk), ("v", vn, dv)):
+        for _ in range(6):
+            idx = tuple(rng.integers(0, s) for s in arr.shape)
+            base = float(np.float32(arr[idx]))
+            args = {"q": qn, "k": kn, "v": vn}
+            plus, minus = arr.copy(), arr.copy()
+            plus[idx], minus[idx] = base + h, base - h
+            lp = loss(*[plus if n == name else args[n] for n in ("q", "k", "v")], kv_in)
+            lm = loss(*[minus if n == name else args[n] for n in ("q", "k", "v")], kv_in)
+            fd = (lp - lm) / (2 * h)  # the loss is linear in each single entry: exact up to rounding
+            assert abs(fd - grad[idx]) <= 1e-9 * max(1.0, abs(grad[idx])), (name, idx, fd, grad[idx])
+    for _ in range(6):
+        idx = tuple(rng.integers(0, s) for s in kv_in.shape)
+        plus, minus = kv_in.copy(), kv_in.copy()
+        plus[idx] += 1e-3
+        minus[idx] -= 1e-3
+        fd = (loss(qn, kn, vn, plus) - loss(qn, kn, vn, minus)) / 2e-3
+        assert abs(fd - gin[idx]) <= 1e-9 * max(1.0, abs(gin[idx]))
+
+
+def test_euler_identities():
+    """O is linear in each of q, k, v, so <Q,dQ> = <K,dK> = <V,dV> = <O,dO> per head."""
+    B, H, N, d, e = 1, 3, 50, 6, 7
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=19)
+    lam = np.array([1.0, 0.95, 0.2])
+    o = orc.fwd_rec(q, k, v, lam)
+    dq, dk, dv = orc.bwd_rec(q, k, v, do, lam)
+    qn, kn, vn, don = (x.double().numpy() for x in (q, k, v, do))
+    ref = np.sum(o * don, axis=(2, 3))
+    for a, b in ((qn, dq), (kn, dk), (vn, dv)):
+        assert np.allclose(np.sum(a * b, axis=(2, 3)), ref, rtol=1e-12)
+
+
+def test_role_swap_identities():
+    """dQ = LA(q:=dO, k:=V, v:=K); dK, dV are the same operator run on the reversed sequence."""
+    B, H, N, d, e = 1, 2, 40, 5, 5
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=23)
+    lam = np.array([0.9, 0.6])
+    dq, dk, dv = orc.bwd_rec(q, k, v, do, lam)
+    assert relerr(orc.fwd_rec(do, v, k, lam), dq) < 1e-13
+    flip = lambda x: torch.flip(x, dims=[2])
+    assert relerr(orc.fwd_rec(flip(v), flip(do), flip(q), lam)[:, :, ::-1], dk) < 1e-13
+    assert relerr(orc.fwd_rec(flip(k), flip(q), flip(do), lam)[:, :, ::-1], dv) < 1e-13
+
+
+def test_linearity_scaling():
+    q, k, v, _ = rand_inputs(1, 1, 20, 4, 4, seed=29)
+    lam = np.array([0.75])
+    base = orc.fwd_rec(q, k, v, lam)
+    assert relerr(orc.fwd_rec(2 * q, 4 * k, 0.5 * v, lam), 4 * base) < 1e-15
+
+
+# --- state hand-over, decode, causality ---------------------------------------------
+@pytest.mark.parametrize("split", [1, 13, 32, 49])
+def test_chaining_equals_one_call(split):
+    B, H, N, d, e = 1, 2, 50, 4, 6
+    q, k, v, _ = rand_inputs(B, H, N, d, e, seed=31)
+    lam = np.array([0.85, 1.0])
+    full, kv_full = orc.fwd_rec(q, k, v, lam, want_state=True)
+    o1, kv1 = orc.fwd_rec(q[:, :, :split], k[:, :, :split], v[:, :, :split], lam, want_state=True)
+    o2, kv2 = orc.fwd_rec(q[:, :, split:], k[:, :, split:], v[:, :, split:], lam, kv_in=kv1, want_state=True)
+    assert relerr(np.concatenate([o1, o2], axis=2), full) < 1e-14
+    assert relerr(kv2, kv_full) < 1e-14
+
+
+def test_decode_steps_equal_parallel_form():
+    B, H, P, S, d, e = 2, 2, 9, 5, 4, 3
+    q, k, v, _ = rand_inputs(B, H, P + S, d, e, seed=37)
+    lam = np.array([0.9, 0.5])
+    full = orc.fwd_quad(q, k, v, lam)
+    _, kv = orc.fwd_rec(q[:, :, :P], k[:, :, :P], v[:, :, :P], lam, want_state=True)
+    for s in range(S):
+        t = P + s
+        o = orc.decode_step(q[:, :, t], k[:, :, t], v[:, :, t], lam, kv)
+        assert relerr(o, full[:, :, t]) < 1e-13
+
+
+def test_causality_bitwise():
+    B, H, N, d, e = 1, 1, 30, 4, 4
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=41)
+    lam = np.array([0.9])
+    t0 = 17
+    q2, k2, v2, do2 = (x.clone() for x in (q, k, v, do))
+    q2[:, :, t0] += 1
+    k2[:, :, t0] -= 2
+    v2[:, :, t0] *= 3
+    o, o2 = orc.fwd_rec(q, k, v, lam), orc.fwd_rec(q2, k2, v2, lam)
+    assert np.array_equal(o[:, :, :t0], o2[:, :, :t0]) and not np.array_equal(o[:, :, t0:], o2[:, :, t0:])
+    dq, _, _ = orc.bwd_rec(q, k, v, do, lam)
+    dqb, _, _ = orc.bwd_rec(q2, k2, v2, do, lam)
+    assert np.array_equal(dq[:, :, :t0], dqb[:, :, :t0])
+    do2[:, :, t0] += 1
+    _, dk, dv = orc.bwd_rec(q, k, v, do, lam)
+    _, dkb, dvb = orc.bwd_rec(q2, k, v, do2, lam)
+    assert np.array_equal(dk[:, :, t0 + 1:], dkb[:, :, t0 + 1:])
+    assert np.array_equal(dv[:, :, t0 + 1:], dvb[:, :, t0 + 1:])
+
+
+# --- the prescaled recurrence: equal while it is safe, broken when it is not ----------
+def test_origin_inference_agrees_then_overflows():
+    q, k, v, _ = rand_inputs(1, 1, 64, 4, 4, seed=43)
+    lam = np.array([0.9])
+    assert relerr(orc.fwd_origin(q, k, v, lam), orc.fwd_rec(q, k, v, lam)) < 1e-10
+    # lambda = e^-2: lambda^-t overflows fp64 once 2 t > ~709
+    q, k, v, _ = rand_inputs(1, 1, 500, 4, 4, seed=43)
+    lam = np.array([np.exp(-2.0)])
+    with np.errstate(all="ignore"):
+        bad = orc.fwd_origin(q, k, v, lam)
+    good = orc.fwd_rec(q, k, v, lam)
+    assert np.all(np.isfinite(good))
+    assert not np.all(np.isfinite(bad[:, :, 400:]))
+
+
+# --- input generator facts ------------------------------------------------------------
+def test_decay_schedule_values():
+    lam = inputs.decay_rates(2, 0.5).double().numpy()
+    assert np.allclose(lam, [1.0, np.exp(-2.0)], rtol=1e-7)
+    lam = inputs.decay_rates(32, 0.9).double().numpy()
+    assert lam[0] == 1.0 and np.allclose(lam[-1], np.exp(-0.025 * 31), rtol=1e-7)
+    lam = inputs.decay_rates(16, 0.25).double().numpy()
+    assert np.allclose(lam[-1], np.exp(-0.375 * 15), rtol=1e-6)
+
+
+def test_generator_is_seeded_and_bf16_exact():
+    a = inputs.make_qkvdo(1, 2, 16, 8, 8, seed=0)
+    b = inputs.make_qkvdo(1, 2, 16, 8, 8, seed=0)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y) and x.dtype == torch.bfloat16
+    # SiLU moments of the draw
+    q = inputs.make_qkvdo(1, 4, 4096, 64, 64, seed=0, dtype=torch.float32)[0]
+    assert abs(q.mean().item() - 0.20662) < 2e-3
+    assert abs((q * q).mean().item() - 0.35578) < 4e-3
