@@ -1,0 +1,164 @@
+/*
+ * la.h -- C ABI of the B200 (sm_100a) library for causal linear attention with
+ * per-head exponential decay.
+ *
+ * What is computed (per batch b and head h, independently):
+ *
+ *   forward   o_t = sum_{s<=t} lambda_h^(t-s) (q_t . k_s) v_s
+ *             i.e. O = (Q K^T (.) M) V with M_ts = lambda^(t-s) for t >= s, else 0
+ *             (Section 3.2.1 "Lightning Attention", Algorithm 3), which equals the
+ *             recurrence kv_t = lambda kv_{t-1} + k_t v_t^T, o_t = kv_t^T q_t
+ *             (Algorithm 2 "Robust Inference"; equivalence: Appendix C).
+ *             No softmax and no 1/sqrt(d) scaling (Section 3.1.4).
+ *   backward  dQ = dA K, dK = dA^T Q, dV = A^T dO with A = (Q K^T) (.) M and
+ *             dA = (dO V^T) (.) M (Algorithm 4), for the loss <O, dO>.
+ *   decode    one iteration of Algorithm 2 on a state kept by the caller.
+ *
+ * Conventions that hold for every entry point
+ *   - Tensors are dense row-major with the feature dimension fastest:
+ *     q,k,dq,dk [B,H,N,d]; v,o,dO,dv [B,H,N,e]; states [B,H,d,e] fp32 with
+ *     kv[b,h,i,j] = sum_s lambda^(t-s) k_s[i] v_s[j].
+ *   - Every tensor pointer is DEVICE memory, 16-byte aligned, owned by the caller.
+ *     The library allocates no device memory, never frees, never synchronises
+ *     the stream and keeps no mutable global state.  Inputs are not modified;
+ *     outputs are fully overwritten; inputs and outputs must not alias (except
+ *     the state of la_decode_step, which is updated in place).
+ *   - `lambda_host` is HOST memory: H floats, each finite and in (0, 1].  It is
+ *     read during the call (validated, converted to -log2(lambda) in double) and
+ *     passed to the kernels by value; it need not outlive the call.
+ *   - All work is enqueued on `stream`; the call returns without waiting.
+ *   - Errors are reported by return code only.  Argument errors are found
+ *     before anything is launched.  There is no CPU fallback: on a device that
+ *     is not sm_100 the calls return LA_ERR_ARCH.
+ *   - Supported in this version: d == e in {64, 128}; H <= 256;
+ *     in_dtype BF16 with out_dtype F32 or BF16, or in = out = F32.
+ *     Accumulation and states are always fp32.
+ */
+#ifndef LA_B200_H
+#define LA_B200_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LA_OK = 0,
+  LA_ERR_INVALID_ARG = 1, /* null/misaligned pointer, bad size, lambda outside (0,1] */
+  LA_ERR_UNSUPPORTED = 2, /* shape or dtype combination not built */
+  LA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than la_workspace_bytes() */
+  LA_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed */
+  LA_ERR_ARCH = 5,        /* current device is not sm_100 */
+  LA_ERR_DEVICE_TIMEOUT = 6 /* a bounded device-side wait expired (see la_read_device_status) */
+} la_status;
+
+typedef enum { LA_BF16 = 0, LA_F32 = 1 } la_dtype;
+
+/* Which kernels run.  AUTO picks the tensor-core kernels where they exist
+ * (bf16 inputs, d = e = 128) and the fp32 CUDA-core kernels otherwise. */
+typedef enum { LA_PATH_AUTO = 0, LA_PATH_SIMT = 1, LA_PATH_TENSOR = 2 } la_path;
+
+/* la_shape.precision, tensor-core path only: bf16 operands formed on chip from fp32
+ * values are carried as two bf16 terms (hi + lo).  Default: both bits set. */
+#define LA_SPLIT_SCORES 1 /* the masked score tile (Q K^T) (.) D                      */
+#define LA_SPLIT_STATE 2  /* the running state used as a matrix operand              */
+#define LA_SPLIT_DECAYED 4 /* the decay-scaled value rows entering the state update  */
+#define LA_PRECISION_DEFAULT (-1)
+
+typedef struct {
+  int B, H, N, d, e;  /* N >= 1 (ignored by la_decode_step) */
+  la_dtype in_dtype;  /* q, k, v, dO */
+  la_dtype out_dtype; /* o, dq, dk, dv */
+  int seg_len;        /* 0 = library chooses.  Otherwise the sequence is cut into
+                         segments of this many tokens (a positive multiple of 128)
+                         that run as independent thread blocks joined by a state scan. */
+  int path;           /* la_path */
+  int precision;      /* LA_PRECISION_DEFAULT or an OR of LA_SPLIT_* */
+} la_shape;
+
+#define LA_OP_FWD 0
+#define LA_OP_BWD 1
+#define LA_OP_DECODE 2
+
+/* Bytes of device scratch the given op needs for this shape (0 is possible).
+ * Returns (size_t)-1 if the shape is invalid or unsupported.  Linear in
+ * B*H*d*e*ceil(N/seg_len); never grows with N^2. */
+size_t la_workspace_bytes(int op, const la_shape* shape);
+
+/* The segment length the library will use for this shape (after applying
+ * shape->seg_len), or 0 if the shape is invalid. */
+int la_segment_length(const la_shape* shape);
+
+/*
+ * Forward pass (Section 3.2.1; Algorithm 3 defines the result, Algorithm 2 the
+ * state).  o [B,H,N,e] <- (Q K^T (.) M) V, optionally continuing from a state:
+ *   kv_in   [B,H,d,e] fp32 state before token 0, or NULL for zeros;
+ *   kv_out  [B,H,d,e] fp32 state after the last token (no extra decay), or NULL.
+ * With kv_in the result is o_t = kv_t^T q_t where kv_{-1} = kv_in.
+ * workspace: device scratch of at least la_workspace_bytes(LA_OP_FWD, shape)
+ * bytes, 256-byte aligned; may be NULL when that size is 0.  Its contents are
+ * undefined afterwards.  Calls that share a workspace must be stream-ordered.
+ */
+la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void* v,
+                 const float* lambda_host, void* o, const float* kv_in, float* kv_out,
+                 void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
+
+/*
+ * Backward pass (Algorithm 4 defines the result): gradients of
+ * L = <O, dO> + <kv_out, grad_kv_out> with respect to q, k, v (and kv_in).
+ *   d_o          [B,H,N,e] in in_dtype;
+ *   dq, dk       [B,H,N,d], dv [B,H,N,e] in out_dtype;
+ *   kv_in        the state given to la_fwd, or NULL;
+ *   grad_kv_out  IN, [B,H,d,e] fp32, dL/d(kv_out), or NULL for zeros;
+ *   grad_kv_in   OUT, [B,H,d,e] fp32, dL/d(kv_in), or NULL if not wanted.
+ * lambda has no gradient (it is not learnable, Section 3.1.1).
+ * workspace as for la_fwd with LA_OP_BWD.
+ */
+la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void* v,
+                 const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
+                 const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
+                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One recurrent decode step (one iteration of Algorithm 2) for every (b,h):
+ *   kv <- lambda_h kv + k v^T   (kv [B,H,d,e] fp32, updated IN PLACE)
+ *   o  <- kv^T q                (o [B,H,e] in out_dtype)
+ * q,k [B,H,d], v [B,H,e] in in_dtype.  shape->N is ignored.  Needs no workspace.
+ * Holds no host state between calls, so a loop of steps may be stream-captured.
+ */
+la_status la_decode_step(const la_shape* shape, const void* q, const void* k, const void* v,
+                         const float* lambda_host, float* kv, void* o, void* stream);
+
+/* Human-readable name of a status code (static string). */
+const char* la_status_string(la_status s);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int la_version(void);
+
+/* Number of kernels this library has launched in the calling process since load
+ * (monotonic counter, relaxed atomics; for benchmarks that report launch counts). */
+unsigned long long la_launch_count(void);
+
+/*
+ * Optional per-kernel timing for benchmarks (no counterpart in the paper).
+ * While enabled, every kernel the library launches is bracketed by a pair of
+ * CUDA events recorded on the caller's stream.  la_profile_collect waits for
+ * those events, adds the elapsed milliseconds and launch counts per kernel kind
+ * into ms[LA_NUM_KERNEL_KINDS] / launches[LA_NUM_KERNEL_KINDS] (both are
+ * overwritten), releases the events and returns LA_OK.  This is the one piece of
+ * mutable process-wide state in the library; it is off by default, guarded by a
+ * mutex, and must not be enabled while a stream is being captured.
+ */
+#define LA_KERNEL_PREPASS 0 /* segment-local states            */
+#define LA_KERNEL_SCAN 1    /* state scan across segments      */
+#define LA_KERNEL_WALK 2    /* block walk producing o/dq/dk/dv */
+#define LA_KERNEL_DECODE 3  /* recurrent decode step           */
+#define LA_NUM_KERNEL_KINDS 4
+void la_profile_enable(int on);
+la_status la_profile_collect(double* ms, unsigned long long* launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LA_B200_H */

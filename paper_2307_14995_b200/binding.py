@@ -1,0 +1,208 @@
+"""Thin ctypes binding of the C ABI in ``include/la.h``.
+
+Argument marshalling only: every step of the attention path runs in the CUDA
+kernels behind ``libla_b200.so``.  PyTorch is used for device memory and streams.
+There is no fallback: if the library is missing or the device is not a B200 the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libla_b200.so")
+
+LA_BF16, LA_F32 = 0, 1
+LA_PATH_AUTO, LA_PATH_SIMT, LA_PATH_TENSOR = 0, 1, 2
+LA_SPLIT_SCORES, LA_SPLIT_STATE, LA_SPLIT_DECAYED = 1, 2, 4
+LA_PRECISION_DEFAULT = -1
+LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
+
+EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
+           "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
+           "la_profile_collect")
+KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
+
+
+class LaShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int), ("H", ctypes.c_int), ("N", ctypes.c_int), ("d", ctypes.c_int),
+                ("e", ctypes.c_int), ("in_dtype", ctypes.c_int), ("out_dtype", ctypes.c_int),
+                ("seg_len", ctypes.c_int), ("path", ctypes.c_int), ("precision", ctypes.c_int)]
+
+
+class LaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s: %s (status %d)" % (where, status_string(code), code))
+
+
+_lib = None
+
+
+def load():
+    """Load the shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing; run `python -m paper_2307_14995_b200.build`"
+                               % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, sz, I = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        sp = ctypes.POINTER(LaShape)
+        fp = ctypes.POINTER(ctypes.c_float)
+        lib.la_workspace_bytes.argtypes = [I, sp]
+        lib.la_workspace_bytes.restype = sz
+        lib.la_segment_length.argtypes = [sp]
+        lib.la_segment_length.restype = I
+        lib.la_fwd.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp, vp, sz, vp]
+        lib.la_fwd.restype = I
+        lib.la_bwd.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.la_bwd.restype = I
+        lib.la_decode_step.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
+        lib.la_decode_step.restype = I
+        lib.la_status_string.argtypes = [I]
+        lib.la_status_string.restype = ctypes.c_char_p
+        lib.la_version.restype = I
+        lib.la_launch_count.restype = ctypes.c_ulonglong
+        lib.la_profile_enable.argtypes = [I]
+        lib.la_profile_enable.restype = None
+        lib.la_profile_collect.argtypes = [ctypes.POINTER(ctypes.c_double),
+                                           ctypes.POINTER(ctypes.c_ulonglong)]
+        lib.la_profile_collect.restype = I
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().la_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(load().la_version())
+
+
+def launch_count() -> int:
+    return int(load().la_launch_count())
+
+
+def profile_enable(on: bool) -> None:
+    load().la_profile_enable(1 if on else 0)
+
+
+def profile_collect():
+    """{kind: (total_ms, launches)} for the kernels launched while profiling was enabled."""
+    ms = (ctypes.c_double * len(KERNEL_KINDS))()
+    n = (ctypes.c_ulonglong * len(KERNEL_KINDS))()
+    rc = load().la_profile_collect(ms, n)
+    if rc != 0:
+        raise LaError(rc, "la_profile_collect")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+_DT = {torch.bfloat16: LA_BF16, torch.float32: LA_F32}
+
+
+def make_shape(B, H, N, d, e, in_dtype, out_dtype, seg_len=0, path=LA_PATH_AUTO,
+               precision=LA_PRECISION_DEFAULT) -> LaShape:
+    return LaShape(B, H, N, d, e, _DT[in_dtype], _DT[out_dtype], seg_len, path, precision)
+
+
+def workspace_bytes(op: int, shape: LaShape) -> int:
+    n = load().la_workspace_bytes(op, ctypes.byref(shape))
+    if n == ctypes.c_size_t(-1).value:
+        raise LaError(2, "la_workspace_bytes")
+    return int(n)
+
+
+def segment_length(shape: LaShape) -> int:
+    return int(load().la_segment_length(ctypes.byref(shape)))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensors must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _lam(lam) -> ctypes.Array:
+    vals = [float(x) for x in (lam.tolist() if hasattr(lam, "tolist") else lam)]
+    return (ctypes.c_float * len(vals))(*vals)
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def alloc_workspace(op: int, shape: LaShape, device) -> Optional[torch.Tensor]:
+    n = workspace_bytes(op, shape)
+    if n == 0:
+        return None
+    return torch.empty(n, dtype=torch.uint8, device=device)  # torch allocations are >= 256-byte aligned
+
+
+def la_fwd(shape: LaShape, q, k, v, lam, o, kv_in=None, kv_out=None, workspace=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_fwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(o), _ptr(kv_in),
+                       _ptr(kv_out), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_fwd")
+
+
+def la_bwd(shape: LaShape, q, k, v, do, lam, dq, dk, dv, kv_in=None, grad_kv_out=None, grad_kv_in=None,
+           workspace=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_bwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(do), _lam(lam), _ptr(dq),
+                       _ptr(dk), _ptr(dv), _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in),
+                       _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_bwd")
+
+
+def la_decode_step(shape: LaShape, q, k, v, lam, kv, o, stream=None):
+    rc = load().la_decode_step(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(kv),
+                               _ptr(o), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_decode_step")
+
+
+# ---- convenience wrappers that allocate outputs with torch -------------------------------
+def fwd(q, k, v, lam, *, out_dtype=torch.float32, kv_in=None, want_state=False, seg_len=0,
+        path=LA_PATH_AUTO, precision=LA_PRECISION_DEFAULT, stream=None):
+    B, H, N, d = q.shape
+    e = v.shape[-1]
+    shape = make_shape(B, H, N, d, e, q.dtype, out_dtype, seg_len, path, precision)
+    o = torch.empty((B, H, N, e), dtype=out_dtype, device=q.device)
+    kv_out = torch.empty((B, H, d, e), dtype=torch.float32, device=q.device) if want_state else None
+    ws = alloc_workspace(LA_OP_FWD, shape, q.device)
+    la_fwd(shape, q, k, v, lam, o, kv_in, kv_out, ws, stream)
+    return (o, kv_out) if want_state else o
+
+
+def bwd(q, k, v, do, lam, *, out_dtype=torch.float32, kv_in=None, grad_kv_out=None,
+        want_state_grad=False, seg_len=0, path=LA_PATH_AUTO, precision=LA_PRECISION_DEFAULT, stream=None):
+    B, H, N, d = q.shape
+    e = v.shape[-1]
+    shape = make_shape(B, H, N, d, e, q.dtype, out_dtype, seg_len, path, precision)
+    dq = torch.empty((B, H, N, d), dtype=out_dtype, device=q.device)
+    dk = torch.empty((B, H, N, d), dtype=out_dtype, device=q.device)
+    dv = torch.empty((B, H, N, e), dtype=out_dtype, device=q.device)
+    gin = torch.empty((B, H, d, e), dtype=torch.float32, device=q.device) if want_state_grad else None
+    ws = alloc_workspace(LA_OP_BWD, shape, q.device)
+    la_bwd(shape, q, k, v, do, lam, dq, dk, dv, kv_in, grad_kv_out, gin, ws, stream)
+    return (dq, dk, dv, gin) if want_state_grad else (dq, dk, dv)
+
+
+def decode_step(q, k, v, lam, kv, *, out_dtype=torch.float32, stream=None):
+    B, H, d = q.shape
+    e = v.shape[-1]
+    shape = make_shape(B, H, 1, d, e, q.dtype, out_dtype)
+    o = torch.empty((B, H, e), dtype=out_dtype, device=q.device)
+    la_decode_step(shape, q, k, v, lam, kv, o, stream)
+    return o

@@ -1,0 +1,354 @@
+// C-ABI entry points (declared in include/la.h): argument validation, the
+// segment plan, workspace carving and the launch sequences.  Nothing here
+// computes attention; every step of the path runs in the kernels.
+#include <atomic>
+#include <mutex>
+#include <vector>
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+
+#include "../../include/la.h"
+#include "la_common.cuh"
+
+namespace la {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// ---- optional benchmark profiling ----------------------------------------------------------
+struct ProfRecord { int kind; cudaEvent_t start, stop; };
+static std::mutex g_prof_mu;
+static std::atomic<bool> g_prof_on{false};
+static std::vector<ProfRecord> g_prof;
+
+KernelTimer::KernelTimer(int kind, cudaStream_t stream)
+    : kind_(kind), stream_(stream), start_(nullptr), active_(false) {
+  if (!g_prof_on.load(std::memory_order_relaxed)) return;
+  if (cudaEventCreate(&start_) != cudaSuccess) return;
+  cudaEventRecord(start_, stream_);
+  active_ = true;
+}
+KernelTimer::~KernelTimer() {
+  if (!active_) return;
+  cudaEvent_t stop;
+  if (cudaEventCreate(&stop) != cudaSuccess) { cudaEventDestroy(start_); return; }
+  cudaEventRecord(stop, stream_);
+  std::lock_guard<std::mutex> lock(g_prof_mu);
+  g_prof.push_back({kind_, start_, stop});
+}
+
+namespace {
+
+struct Plan {
+  int BH, seg_len, nseg;
+  bool tensor;      // tensor-core kernels
+  int precision;    // LA_SPLIT_* bits (tensor path)
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+la_status check_shape(const la_shape* s, bool need_n) {
+  if (!s) return LA_ERR_INVALID_ARG;
+  if (s->B < 1 || s->H < 1 || s->d < 1 || s->e < 1) return LA_ERR_INVALID_ARG;
+  if (need_n && s->N < 1) return LA_ERR_INVALID_ARG;
+  if (s->in_dtype != LA_BF16 && s->in_dtype != LA_F32) return LA_ERR_INVALID_ARG;
+  if (s->out_dtype != LA_BF16 && s->out_dtype != LA_F32) return LA_ERR_INVALID_ARG;
+  if (s->seg_len < 0 || (s->seg_len % 128) != 0) return LA_ERR_INVALID_ARG;
+  if (s->path < LA_PATH_AUTO || s->path > LA_PATH_TENSOR) return LA_ERR_INVALID_ARG;
+  if (s->precision != LA_PRECISION_DEFAULT && (s->precision < 0 || s->precision > 7))
+    return LA_ERR_INVALID_ARG;
+  if (s->H > LA_MAX_H) return LA_ERR_UNSUPPORTED;
+  if (!(s->d == s->e && (s->d == 64 || s->d == 128))) return LA_ERR_UNSUPPORTED;
+  if (s->in_dtype == LA_F32 && s->out_dtype != LA_F32) return LA_ERR_UNSUPPORTED;
+  // element counts must fit the 32-bit coordinates the kernels and tensor maps use
+  const double tokens = (double)s->B * s->H * (need_n ? s->N : 1);
+  if (tokens * s->d >= 2147483648.0 * 64.0 || (double)s->B * s->H >= 2147483648.0 ||
+      (need_n && (double)s->N >= 1073741824.0))
+    return LA_ERR_UNSUPPORTED;
+  return LA_OK;
+}
+
+bool tensor_path_available(const la_shape* s) {
+  return tc_supported() && s->in_dtype == LA_BF16 && s->d == 128 && s->e == 128;
+}
+
+la_status make_plan(const la_shape* s, Plan* p) {
+  p->BH = s->B * s->H;
+  if (s->path == LA_PATH_TENSOR && !tensor_path_available(s)) return LA_ERR_UNSUPPORTED;
+  p->tensor = (s->path == LA_PATH_TENSOR) || (s->path == LA_PATH_AUTO && tensor_path_available(s));
+  p->precision = (s->precision == LA_PRECISION_DEFAULT)
+                     ? (LA_SPLIT_SCORES | LA_SPLIT_STATE | LA_SPLIT_DECAYED)
+                     : s->precision;
+  long seg_len = s->seg_len;
+  if (seg_len == 0) {
+    // Enough independent thread blocks to cover the 148 SMs a few times over, but
+    // segments no shorter than 1024 tokens so the per-segment state traffic stays small.
+    const long target = 592;
+    const long slices = p->tensor ? 2 : 1;  // the tensor kernels also split the value columns
+    long want = (target + p->BH * slices - 1) / (p->BH * slices);
+    long most = s->N / 1024;
+    if (most < 1) most = 1;
+    if (want > most) want = most;
+    if (want < 1) want = 1;
+    seg_len = (s->N + want - 1) / want;
+    seg_len = (seg_len + 127) / 128 * 128;
+  }
+  p->seg_len = (int)seg_len;
+  p->nseg = (int)((s->N + seg_len - 1) / seg_len);
+  return LA_OK;
+}
+
+size_t state_set_bytes(const la_shape* s, const Plan& p) {
+  return (size_t)p.BH * p.nseg * s->d * s->e * sizeof(float);
+}
+
+la_status make_table(const la_shape* s, const float* lambda_host, DecayTable* tab) {
+  if (!lambda_host) return LA_ERR_INVALID_ARG;
+  for (int h = 0; h < s->H; ++h) {
+    const float lam = lambda_host[h];
+    if (!(std::isfinite(lam) && lam > 0.f && lam <= 1.f)) return LA_ERR_INVALID_ARG;
+    const double s2 = -std::log2((double)lam);
+    tab->s2[h] = (s2 > 0.0) ? s2 : 0.0;  // lambda == 1 gives exactly 0 (never -0)
+  }
+  for (int h = s->H; h < LA_MAX_H; ++h) tab->s2[h] = 0.0;
+  return LA_OK;
+}
+
+la_status check_device() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LA_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return LA_ERR_CUDA;
+  return major == 10 ? LA_OK : LA_ERR_ARCH;
+}
+
+#define LA_TRY_CUDA(expr)                       \
+  do {                                          \
+    if ((expr) != cudaSuccess) return LA_ERR_CUDA; \
+  } while (0)
+
+// One generic-operator call: optional pre-pass + scan (when the sequence is cut
+// into segments or the incoming state needs transposing), then the walk.
+struct OpCall {
+  const void *a, *b, *c;
+  void* out;
+  int reverse;
+  const float* z_in;     // user state entering the sequence (kernel orientation unless transposed)
+  bool z_in_transposed;
+  float* final_out;      // state leaving the sequence, kernel orientation, or NULL
+  float* buf;            // [BH,nseg,D*E] scratch for entry states (may be NULL if not needed)
+};
+
+cudaError_t run_prepass(const la_shape* s, const Plan& p, const DecayTable& tab, const void* b,
+                        const void* c, int reverse, float* local_out, cudaStream_t st) {
+  OpArgs args{};
+  args.b = b;
+  args.c = c;
+  args.local_out = local_out;
+  args.BH = p.BH;
+  args.H = s->H;
+  args.N = s->N;
+  args.seg_len = p.seg_len;
+  args.nseg = p.nseg;
+  args.reverse = reverse;
+  if (p.tensor) return launch_tc_prepass(args, tab, p.precision, st);
+  return launch_simt_prepass(args, tab, s->d, s->e, (int)s->in_dtype, st);
+}
+
+cudaError_t run_scan(const la_shape* s, const Plan& p, const DecayTable& tab, float* buf, float* buf_t,
+                     const float* z_in, bool z_in_transposed, int reverse, cudaStream_t st) {
+  ScanArgs sa{};
+  sa.buf = buf;
+  sa.buf_t = buf_t;
+  sa.z_in = z_in;
+  sa.z_in_transposed = z_in_transposed ? 1 : 0;
+  sa.BH = p.BH;
+  sa.H = s->H;
+  sa.N = s->N;
+  sa.seg_len = p.seg_len;
+  sa.nseg = p.nseg;
+  sa.Da = s->d;  // d == e in every supported shape, so both orientations are square
+  sa.Ec = s->e;
+  sa.reverse = reverse;
+  return launch_scan(sa, tab, st);
+}
+
+cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, const void* a,
+                     const void* b, const void* c, void* out, const float* entry, float* final_out,
+                     int reverse, cudaStream_t st) {
+  OpArgs args{};
+  args.a = a;
+  args.b = b;
+  args.c = c;
+  args.out = out;
+  args.entry = entry;
+  args.final_out = final_out;
+  args.BH = p.BH;
+  args.H = s->H;
+  args.N = s->N;
+  args.seg_len = p.seg_len;
+  args.nseg = p.nseg;
+  args.reverse = reverse;
+  if (p.tensor) return launch_tc_walk(args, tab, (int)s->out_dtype, p.precision, st);
+  return launch_simt_walk(args, tab, s->d, s->e, (int)s->in_dtype, (int)s->out_dtype, st);
+}
+
+}  // namespace
+}  // namespace la
+
+using namespace la;
+
+extern "C" {
+
+size_t la_workspace_bytes(int op, const la_shape* shape) {
+  if (op != LA_OP_FWD && op != LA_OP_BWD && op != LA_OP_DECODE) return (size_t)-1;
+  if (check_shape(shape, op != LA_OP_DECODE) != LA_OK) return (size_t)-1;
+  if (op == LA_OP_DECODE) return 0;
+  Plan p;
+  if (make_plan(shape, &p) != LA_OK) return (size_t)-1;
+  const size_t one = state_set_bytes(shape, p);
+  if (op == LA_OP_FWD) return p.nseg > 1 ? one : 0;
+  return 3 * one;
+}
+
+int la_segment_length(const la_shape* shape) {
+  if (check_shape(shape, true) != LA_OK) return 0;
+  Plan p;
+  if (make_plan(shape, &p) != LA_OK) return 0;
+  return p.seg_len;
+}
+
+la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void* v,
+                 const float* lambda_host, void* o, const float* kv_in, float* kv_out,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+  la_status st = check_shape(shape, true);
+  if (st != LA_OK) return st;
+  if (!q || !k || !v || !o) return LA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(kv_in) ||
+      !aligned16(kv_out))
+    return LA_ERR_INVALID_ARG;
+  DecayTable tab;
+  if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
+  Plan p;
+  if ((st = make_plan(shape, &p)) != LA_OK) return st;
+  const size_t need = p.nseg > 1 ? state_set_bytes(shape, p) : 0;
+  if (need > 0 && (!workspace || workspace_bytes < need)) return LA_ERR_WORKSPACE;
+  if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return LA_ERR_INVALID_ARG;
+  if ((st = check_device()) != LA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+  const float* entry = kv_in;  // single segment: the caller's state is the entry state
+  if (p.nseg > 1) {
+    float* buf = static_cast<float*>(workspace);
+    LA_TRY_CUDA(run_prepass(shape, p, tab, k, v, 0, buf, cs));
+    LA_TRY_CUDA(run_scan(shape, p, tab, buf, nullptr, kv_in, false, 0, cs));
+    entry = buf;
+  }
+  LA_TRY_CUDA(run_walk(shape, p, tab, q, k, v, o, entry, kv_out, 0, cs));
+  return LA_OK;
+}
+
+la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void* v,
+                 const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
+                 const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+  la_status st = check_shape(shape, true);
+  if (st != LA_OK) return st;
+  if (!q || !k || !v || !d_o || !dq || !dk || !dv) return LA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
+      !aligned16(dk) || !aligned16(dv) || !aligned16(kv_in) || !aligned16(grad_kv_out) ||
+      !aligned16(grad_kv_in))
+    return LA_ERR_INVALID_ARG;
+  DecayTable tab;
+  if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
+  Plan p;
+  if ((st = make_plan(shape, &p)) != LA_OK) return st;
+  const size_t one = state_set_bytes(shape, p);
+  if (!workspace || workspace_bytes < 3 * one) return LA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LA_ERR_INVALID_ARG;
+  if ((st = check_device()) != LA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+  float* buf_kvt = static_cast<float*>(workspace);                 // KV^T entering each segment
+  float* buf_e = buf_kvt + one / sizeof(float);                    // dKV entering each segment (from the right)
+  float* buf_et = buf_e + one / sizeof(float);                     // its transpose
+  const bool multi = p.nseg > 1;
+
+  // dQ = fwd(a = dO, b = V, c = K); its state is KV^T, so the caller's kv_in enters transposed.
+  const float* entry_q = nullptr;
+  if (multi) LA_TRY_CUDA(run_prepass(shape, p, tab, v, k, 0, buf_kvt, cs));
+  if (multi || kv_in) {
+    LA_TRY_CUDA(run_scan(shape, p, tab, buf_kvt, nullptr, kv_in, true, 0, cs));
+    entry_q = buf_kvt;
+  }
+  LA_TRY_CUDA(run_walk(shape, p, tab, d_o, v, k, dq, entry_q, nullptr, 0, cs));
+
+  // dV = rev(a = K, b = Q, c = dO) carries dKV; dK = rev(a = V, b = dO, c = Q) carries dKV^T.
+  const float* entry_v = nullptr;
+  const float* entry_k = nullptr;
+  if (multi) LA_TRY_CUDA(run_prepass(shape, p, tab, q, d_o, 1, buf_e, cs));
+  if (multi || grad_kv_out) {
+    LA_TRY_CUDA(run_scan(shape, p, tab, buf_e, buf_et, grad_kv_out, false, 1, cs));
+    entry_v = buf_e;
+    entry_k = buf_et;
+  }
+  LA_TRY_CUDA(run_walk(shape, p, tab, k, q, d_o, dv, entry_v, grad_kv_in, 1, cs));
+  LA_TRY_CUDA(run_walk(shape, p, tab, v, d_o, q, dk, entry_k, nullptr, 1, cs));
+  return LA_OK;
+}
+
+la_status la_decode_step(const la_shape* shape, const void* q, const void* k, const void* v,
+                         const float* lambda_host, float* kv, void* o, void* stream) {
+  la_status st = check_shape(shape, false);
+  if (st != LA_OK) return st;
+  if (!q || !k || !v || !kv || !o) return LA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(kv) || !aligned16(o))
+    return LA_ERR_INVALID_ARG;
+  DecayTable tab;
+  if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
+  if ((st = check_device()) != LA_OK) return st;
+  LA_TRY_CUDA(launch_decode(q, k, v, kv, o, shape->B * shape->H, shape->H, shape->d, shape->e,
+                            (int)shape->in_dtype, (int)shape->out_dtype, tab,
+                            static_cast<cudaStream_t>(stream)));
+  return LA_OK;
+}
+
+const char* la_status_string(la_status s) {
+  switch (s) {
+    case LA_OK: return "ok";
+    case LA_ERR_INVALID_ARG: return "invalid argument";
+    case LA_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case LA_ERR_WORKSPACE: return "workspace missing or too small";
+    case LA_ERR_CUDA: return "CUDA call or launch failed";
+    case LA_ERR_ARCH: return "device is not sm_100";
+    case LA_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+  }
+  return "unknown status";
+}
+
+int la_version(void) { return 100; }
+
+void la_profile_enable(int on) { g_prof_on.store(on != 0, std::memory_order_relaxed); }
+
+la_status la_profile_collect(double* ms, unsigned long long* launches) {
+  if (!ms || !launches) return LA_ERR_INVALID_ARG;
+  for (int i = 0; i < LA_NUM_KERNEL_KINDS; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  std::lock_guard<std::mutex> lock(g_prof_mu);
+  la_status st = LA_OK;
+  for (const ProfRecord& r : g_prof) {
+    float t = 0.f;
+    if (cudaEventSynchronize(r.stop) != cudaSuccess ||
+        cudaEventElapsedTime(&t, r.start, r.stop) != cudaSuccess)
+      st = LA_ERR_CUDA;
+    if (r.kind >= 0 && r.kind < LA_NUM_KERNEL_KINDS) { ms[r.kind] += t; launches[r.kind] += 1; }
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  g_prof.clear();
+  return st;
+}
+
+unsigned long long la_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,116 @@
+// Shared declarations of the CUDA side: kernel parameter blocks and the launch
+// helpers that the C-ABI entry points in la_api.cu call.
+//
+// One generic operator covers forward and all three gradients.  With a
+// "query-like" a [N,Da], a "key-like" b [N,Da] and a "value-like" c [N,Ec]:
+//
+//   forward direction   out_t = sum_{s<=t} lambda^(t-s) (a_t.b_s) c_s + lambda^(t+1)   Z_in^T a_t
+//   reverse direction   out_t = sum_{s>=t} lambda^(s-t) (a_t.b_s) c_s + lambda^(N-1-t) Z_in^T a_t
+//
+// where Z is the Da x Ec running state sum_s decay * b_s c_s^T.  Then
+//   O  = fwd(a=Q,  b=K,  c=V)        state = KV          (Algorithm 2 / Algorithm 3)
+//   dQ = fwd(a=dO, b=V,  c=K)        state = KV^T        (Algorithm 4, dQ line)
+//   dK = rev(a=V,  b=dO, c=Q)        state = (dKV)^T     (Algorithm 4, dK line)
+//   dV = rev(a=K,  b=Q,  c=dO)       state = dKV         (Algorithm 4, dV line)
+// The sequence is processed in blocks of C tokens (block-local index i, j):
+//   out_blk = ((a b^T) (.) D) c + diag(f_out) a Z,      Z <- Gamma Z + b^T diag(f_state) c
+// with every decay factor a non-negative power of lambda:
+//   forward: D_ij = lambda^(i-j) [i>=j], f_out_i = lambda^(i+1),    f_state_j = lambda^(Cr-1-j)
+//   reverse: D_ij = lambda^(j-i) [j>=i], f_out_i = lambda^(Cr-1-i), f_state_j = lambda^(j+1)
+//   Gamma = lambda^Cr, Cr = number of real tokens in the block (a ragged last block
+//   uses its own Cr so that no state is decayed through padding).
+// Factors are evaluated as exp2(-s2 * n) with s2 = -log2(lambda) >= 0, never as a
+// ratio of powers, so nothing can overflow and underflow only flushes to the
+// correct limit 0 (this is what the prescaled form of Algorithm 1 cannot offer).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#define LA_MAX_H 256
+
+namespace la {
+
+struct DecayTable {
+  double s2[LA_MAX_H];  // -log2(lambda_h) >= 0, computed in double on the host
+};
+
+// Arguments of one generic-operator launch (either the walking kernel or the
+// state-only pre-pass).
+struct OpArgs {
+  const void* a;      // [BH, N, Da]  (unused by the pre-pass)
+  const void* b;      // [BH, N, Da]
+  const void* c;      // [BH, N, Ec]
+  void* out;          // [BH, N, Ec]  (unused by the pre-pass)
+  const float* entry; // [BH, nseg, Da*Ec] state entering each segment, or NULL = zeros
+  float* local_out;   // pre-pass: [BH, nseg, Da*Ec] segment-local states
+  float* final_out;   // [BH, Da*Ec] state leaving the last-processed segment, or NULL
+  int BH, H, N;
+  int seg_len, nseg;  // seg_len is a multiple of 128
+  int reverse;        // 0 forward, 1 reverse
+};
+
+struct ScanArgs {
+  float* buf;          // [BH, nseg, Da*Ec]: in = segment-local states, out = entry states
+  float* buf_t;        // optional transposed copy of the entry states [BH, nseg, Ec*Da]
+  const float* z_in;   // [BH, Da*Ec] (or [BH, Ec*Da] if z_in_transposed), or NULL = zeros
+  int z_in_transposed;
+  int BH, H, N, seg_len, nseg, Da, Ec, reverse;
+};
+
+// dtype tags as in la.h
+enum { DT_BF16 = 0, DT_F32 = 1 };
+
+// Each returns cudaGetLastError() of its launch.
+cudaError_t launch_simt_walk(const OpArgs& args, const DecayTable& tab, int Da, int Ec, int in_dt,
+                             int out_dt, cudaStream_t stream);
+cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int Da, int Ec, int in_dt,
+                                cudaStream_t stream);
+cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream);
+cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv, void* o, int BH,
+                          int H, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
+                          cudaStream_t stream);
+
+// Tensor-core (tcgen05) kernels: bf16 inputs, Da = Ec = 128.
+bool tc_supported();
+cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int out_dt, int precision,
+                           cudaStream_t stream);
+cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int precision,
+                              cudaStream_t stream);
+
+void count_launch(int n = 1);
+
+// Brackets one kernel launch with CUDA events when benchmark profiling is enabled
+// (la_profile_enable); otherwise does nothing.  kind is one of LA_KERNEL_*.
+struct KernelTimer {
+  KernelTimer(int kind, cudaStream_t stream);
+  ~KernelTimer();
+  int kind_;
+  cudaStream_t stream_;
+  cudaEvent_t start_;
+  bool active_;
+};
+enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_NUM = 4 };
+
+// ---- small device helpers --------------------------------------------------
+__device__ __forceinline__ float decay_pow(float s2, float n) {
+  // lambda^n for n >= 0; s2 == 0 (lambda == 1) gives exactly 1.
+  return exp2f(-s2 * n);
+}
+__device__ __forceinline__ float decay_pow_d(double s2, double n) {
+  // Same in double, rounded once; used where a handful of factors per block are tabulated.
+  return (float)exp2(-s2 * n);
+}
+
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) {
+  return __bfloat162float(x);
+}
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+}  // namespace la

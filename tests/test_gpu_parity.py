@@ -1,0 +1,391 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 CPU oracle.
+
+Tolerances (per tensor and per (b,h) slice, which is the stricter reading):
+  bf16 inputs, fp32 accumulation:  max|err| <= 2e-2 * RMS(ref)
+  fp32 workload:                   max|err| <= 1e-4 * RMS(ref)
+bf16 *outputs* add the output rounding itself: |err| <= 2e-2*RMS + 2^-8*|ref|.
+"""
+import numpy as np
+import pytest
+import torch
+
+from la_check import TOL_BF16, TOL_F32, assert_close, head_err
+from oracle import la_oracle as orc
+from paper_2307_14995_b200 import binding as la, inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+PATHS = [la.LA_PATH_SIMT, la.LA_PATH_TENSOR]
+
+
+def path_ok(path, d, dtype):
+    if path == la.LA_PATH_TENSOR:
+        s = la.make_shape(1, 1, 128, d, d, dtype, torch.float32, 0, path)
+        try:
+            la.workspace_bytes(la.LA_OP_FWD, s)
+        except la.LaError:
+            return False
+    return True
+
+
+def to_dev(*xs):
+    return [None if x is None else x.to(DEV) for x in xs]
+
+
+def fwd_bwd_gpu(q, k, v, do, lam, *, out_dtype=torch.float32, kv_in=None, gko=None, seg_len=0,
+                path=la.LA_PATH_AUTO, precision=la.LA_PRECISION_DEFAULT):
+    qg, kg, vg, dog, kin, gk = to_dev(q, k, v, do, kv_in, gko)
+    o, kv = la.fwd(qg, kg, vg, lam, out_dtype=out_dtype, kv_in=kin, want_state=True, seg_len=seg_len,
+                   path=path, precision=precision)
+    dq, dk, dv, gin = la.bwd(qg, kg, vg, dog, lam, out_dtype=out_dtype, kv_in=kin, grad_kv_out=gk,
+                             want_state_grad=True, seg_len=seg_len, path=path, precision=precision)
+    torch.cuda.synchronize()
+    return o, kv, dq, dk, dv, gin
+
+
+def oracle_all(q, k, v, do, lam, kv_in=None, gko=None):
+    lam64 = lam.double().numpy()
+    o, kv = orc.fwd_rec(q, k, v, lam64, kv_in=kv_in, want_state=True)
+    dq, dk, dv, gin = orc.bwd_rec(q, k, v, do, lam64, kv_in=kv_in, grad_kv_out=gko, want_state_grad=True)
+    return o, kv, dq, dk, dv, gin
+
+
+NAMES = ("o", "kv_out", "dq", "dk", "dv", "grad_kv_in")
+
+
+def compare_all(got, ref, tol):
+    worst = 0.0
+    for n, g, r in zip(NAMES, got, ref):
+        worst = max(worst, assert_close(g, r, tol, n))
+    return worst
+
+
+# ---- the five benchmark workloads -----------------------------------------------------------
+def test_workload_pr1_fp32():
+    w = inputs.make_workload("pr1_ref")
+    got = fwd_bwd_gpu(w["q"], w["k"], w["v"], w["do"], w["lam"])
+    ref = oracle_all(w["q"], w["k"], w["v"], w["do"], w["lam"])
+    compare_all(got, ref, TOL_F32)
+    # and against the masked quadratic form itself
+    lam64 = w["lam"].double().numpy()
+    assert_close(got[0], orc.fwd_quad(w["q"], w["k"], w["v"], lam64), TOL_F32, "o vs quad")
+    for n, g, r in zip(("dq", "dk", "dv"), got[2:5], orc.bwd_quad(w["q"], w["k"], w["v"], w["do"], lam64)):
+        assert_close(g, r, TOL_F32, n + " vs quad")
+
+
+def sample_rows(BH, N, per_head, rng, always=(0,)):
+    bh, t = [], []
+    for x in range(BH):
+        ts = set(int(a) for a in always if a < N) | {N - 1}
+        while len(ts) < min(per_head, N):
+            ts.add(int(rng.integers(0, N)))
+        for a in sorted(ts):
+            bh.append(x)
+            t.append(a)
+    return np.array(bh, np.int32), np.array(t, np.int32)
+
+
+def check_rows(q, k, v, do, lam, got, per_head, tol, seed=0, always=(0, 127, 128)):
+    """Sampled rows of the quadratic form against the GPU tensors (o, dq, dk, dv)."""
+    B, H, N, _ = q.shape
+    rng = np.random.default_rng(seed)
+    lam64 = lam.double().numpy()
+    # RMS per head comes from the GPU tensor itself here (the oracle sees only the sampled rows)
+    for kind, g in zip(("o", "dq", "dk", "dv"), got):
+        bh, t = sample_rows(B * H, N, per_head, rng, always)
+        ref = orc.rows(kind, q, k, v, do, lam64, bh, t)
+        g2 = g.reshape(B * H, N, -1)
+        rms = torch.sqrt(torch.mean(g2.double() ** 2, dim=(1, 2))).cpu().numpy()
+        sel = g2[torch.from_numpy(bh).long().to(g.device), torch.from_numpy(t).long().to(g.device)]
+        err = np.max(np.abs(sel.double().cpu().numpy() - ref), axis=1) / rms[bh]
+        assert np.all(np.isfinite(err)) and err.max() <= tol, (kind, err.max())
+
+
+def test_workload_385m_bf16():
+    w = inputs.make_workload("385m")
+    got = fwd_bwd_gpu(w["q"], w["k"], w["v"], w["do"], w["lam"])
+    ref = oracle_all(w["q"], w["k"], w["v"], w["do"], w["lam"])
+    compare_all(got, ref, TOL_BF16)
+    check_rows(w["q"], w["k"], w["v"], w["do"], w["lam"], (got[0], got[2], got[3], got[4]), 3, TOL_BF16)
+
+
+def test_workload_1b_bf16():
+    w = inputs.make_workload("1b")
+    got = fwd_bwd_gpu(w["q"], w["k"], w["v"], w["do"], w["lam"])
+    ref = oracle_all(w["q"], w["k"], w["v"], w["do"], w["lam"])
+    compare_all(got, ref, TOL_BF16)
+    check_rows(w["q"], w["k"], w["v"], w["do"], w["lam"], (got[0], got[2], got[3], got[4]), 3, TOL_BF16)
+
+
+def test_workload_7b_long_full_size_sampled():
+    """Full-size launch configuration (B=1, H=32, N=65536, d=128); inputs drawn on the GPU from the
+    workload's distributions, the oracle checks whole heads (recurrence) and sampled rows
+    (quadratic form), and the Euler identities tie every head's full tensors together."""
+    w = inputs.device_randn_like_workload("7b_long", DEV, seed=0)
+    q, k, v, do, lam = w["q"], w["k"], w["v"], w["do"], w["lam"]
+    o = la.fwd(q, k, v, lam)
+    dq, dk, dv = la.bwd(q, k, v, do, lam)
+    torch.cuda.synchronize()
+    heads = [0, 1, 13, 31]
+    qs, ks, vs, dos = (x[:, heads].cpu() for x in (q, k, v, do))
+    lam_s = lam[heads]
+    ref = oracle_all(qs, ks, vs, dos, lam_s)
+    for n, g, r in zip(("o", "dq", "dk", "dv"), (o, dq, dk, dv), (ref[0], ref[2], ref[3], ref[4])):
+        assert_close(g[:, heads], r, TOL_BF16, n)
+    rows_heads = [2, 7, 20, 26]
+    qs, ks, vs, dos = (x[:, rows_heads].cpu() for x in (q, k, v, do))
+    check_rows(qs, ks, vs, dos, lam[rows_heads], [x[:, rows_heads] for x in (o, dq, dk, dv)], 4, TOL_BF16,
+               always=(0, 128, 4095, 4096))
+    # <Q,dQ> = <K,dK> = <V,dV> = <O,dO> per head
+    dots = [torch.sum(a.double() * b.double(), dim=(2, 3)) for a, b in ((o, do), (q, dq), (k, dk), (v, dv))]
+    scale = torch.sqrt(torch.sum(o.double() ** 2, dim=(2, 3)) * torch.sum(do.double() ** 2, dim=(2, 3)))
+    for x in dots[1:]:
+        assert torch.all(torch.abs(x - dots[0]) <= 1e-3 * scale)
+
+
+@pytest.mark.parametrize("B,steps", [(8, 256), (64, 32)])
+def test_workload_decode(B, steps):
+    """Prefill 4096 tokens with la_fwd (state out), then recurrent steps; outputs checked against
+    the parallel form over all prefill+steps tokens.  B=64 is the benchmark's launch configuration
+    (GPU-drawn inputs, sampled (b,h)); B=8 runs all 256 steps with CPU-drawn inputs."""
+    H, P, d = 32, 4096, 128
+    if B == 8:
+        x = inputs.make_decode_inputs("decode", B=B, steps=steps)
+        q, k, v, qs, ks, vs, lam = (x[n] for n in ("q", "k", "v", "qs", "ks", "vs", "lam"))
+        qg, kg, vg, qsg, ksg, vsg = to_dev(q, k, v, qs, ks, vs)
+        check_bh = list(range(B * H))
+    else:
+        w = inputs.WORKLOADS["decode"]
+        gen = torch.Generator(DEV)
+        gen.manual_seed(0)
+        silu = lambda s: torch.nn.functional.silu(torch.randn(s, generator=gen, device=DEV)).to(torch.bfloat16)
+        normal = lambda s: torch.randn(s, generator=gen, device=DEV).to(torch.bfloat16)
+        qg, kg, vg = silu((B, H, P, d)), silu((B, H, P, d)), normal((B, H, P, d))
+        qsg, ksg, vsg = silu((steps, B, H, d)), silu((steps, B, H, d)), normal((steps, B, H, d))
+        lam = inputs.decay_rates(w.H, w.l_over_L)
+        check_bh = [0, 31, 32 * 17 + 5, 32 * 40 + 13, B * H - 1]
+    _, kv = la.fwd(qg, kg, vg, lam, want_state=True)
+    outs = []
+    for s in range(steps):
+        outs.append(la.decode_step(qsg[s], ksg[s], vsg[s], lam, kv))
+    torch.cuda.synchronize()
+    out = torch.stack(outs, dim=2)  # [B,H,steps,e]
+    # oracle on the selected (b,h): full sequences of P+steps tokens
+    def gather(pre, st):
+        pre2 = pre.reshape(B * H, P, d)[check_bh].cpu()
+        st2 = st.permute(1, 2, 0, 3).reshape(B * H, steps, d)[check_bh].cpu()
+        return torch.cat([pre2, st2], dim=1).unsqueeze(0)  # [1, nsel, P+steps, d]
+    qf, kf, vf = gather(qg, qsg), gather(kg, ksg), gather(vg, vsg)
+    lam_sel = lam[[x % H for x in check_bh]].double().numpy()
+    # the oracle treats the selected slices as heads of one batch entry
+    ref_o, ref_kv = orc.fwd_rec(qf, kf, vf, lam_sel, want_state=True)
+    got = out.reshape(B * H, steps, d)[check_bh].unsqueeze(0)
+    assert_close(got, ref_o[:, :, P:], TOL_BF16, "decode outputs vs recurrence")
+    assert_close(kv.reshape(B * H, d, d)[check_bh].unsqueeze(0), ref_kv, TOL_BF16, "final state")
+    # the parallel (quadratic) form on sampled rows t >= P
+    rng = np.random.default_rng(0)
+    nsel = len(check_bh)
+    pick = rng.choice(nsel, size=min(nsel, 8), replace=False)
+    bh = np.repeat(pick, 3).astype(np.int32)
+    t = np.concatenate([[P, P + steps - 1, P + int(rng.integers(0, steps))] for _ in pick]).astype(np.int32)
+    rows = orc.rows("o", qf, kf, vf, None, lam_sel, bh, t)
+    rms = np.sqrt(np.mean(ref_o[0] ** 2, axis=(1, 2)))
+    g = got[0].double().cpu().numpy()[bh, t - P]
+    assert np.max(np.max(np.abs(g - rows), axis=1) / rms[bh]) <= TOL_BF16
+
+
+# ---- shapes: tiny, ragged, multi-segment, with state hand-over ----------------------------------
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("N", [1, 2, 31, 33, 127, 128, 129, 257, 1000])
+def test_ragged_lengths_with_states(N, d, path):
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H = 2, 3
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=N)
+    lam = torch.tensor([1.0, 0.97, 0.3])
+    kv_in = inputs.make_state(B, H, d, d, seed=5)
+    gko = inputs.make_state(B, H, d, d, seed=6)
+    ref = oracle_all(q, k, v, do, lam, kv_in.double().numpy(), gko.double().numpy())
+    for seg_len in (0, 128):
+        got = fwd_bwd_gpu(q, k, v, do, lam, kv_in=kv_in, gko=gko, seg_len=seg_len, path=path)
+        compare_all(got, ref, TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_no_states_multi_segment(path):
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N = 1, 4, 700
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=2)
+    lam = inputs.decay_rates(4, 0.5)
+    ref = oracle_all(q, k, v, do, lam)
+    for seg_len in (0, 128, 256):
+        got = fwd_bwd_gpu(q, k, v, do, lam, seg_len=seg_len, path=path)
+        compare_all(got, ref, TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_bf16_outputs(path):
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N = 1, 4, 600
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=3)
+    lam = inputs.decay_rates(4, 0.5)
+    ref = oracle_all(q, k, v, do, lam)
+    got = fwd_bwd_gpu(q, k, v, do, lam, out_dtype=torch.bfloat16, seg_len=256, path=path)
+    for n, g, r in zip(("o", "dq", "dk", "dv"), (got[0], got[2], got[3], got[4]), (ref[0], ref[2], ref[3], ref[4])):
+        assert g.dtype == torch.bfloat16
+        gn = g.double().cpu().numpy().reshape(B * H, -1)
+        rn = r.reshape(B * H, -1)
+        rms = np.sqrt(np.mean(rn * rn, axis=1, keepdims=True))
+        assert np.all(np.abs(gn - rn) <= TOL_BF16 * rms + 2.0 ** -8 * np.abs(rn)), n
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("lam_val", [1.0, 1e-30])
+def test_limits_no_decay_and_instant_decay(lam_val, path):
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N = 1, 2, 300
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=4)
+    lam = torch.tensor([lam_val, lam_val])
+    got = fwd_bwd_gpu(q, k, v, do, lam, seg_len=128, path=path)
+    ref = oracle_all(q, k, v, do, lam)
+    compare_all(got, ref, TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4)
+    if lam_val < 1e-20:  # o_t = (q_t.k_t) v_t
+        qk = (q.double() * k.double()).sum(-1, keepdim=True)
+        assert_close(got[0], (qk * v.double()).numpy(), TOL_BF16, "diagonal limit")
+
+
+# ---- chaining, decode consistency, determinism, guard bands, causality ----------------------------
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("split", [1, 100, 128, 391])
+def test_chaining_equals_one_call(split, path):
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N = 1, 2, 500
+    q, k, v, _ = inputs.make_qkvdo(B, H, N, d, d, seed=8)
+    lam = torch.tensor([0.99, 0.8])
+    qg, kg, vg = to_dev(q, k, v)
+    full, kv_full = la.fwd(qg, kg, vg, lam, want_state=True, path=path)
+    o1, kv1 = la.fwd(qg[:, :, :split].contiguous(), kg[:, :, :split].contiguous(),
+                     vg[:, :, :split].contiguous(), lam, want_state=True, path=path)
+    o2, kv2 = la.fwd(qg[:, :, split:].contiguous(), kg[:, :, split:].contiguous(),
+                     vg[:, :, split:].contiguous(), lam, kv_in=kv1, want_state=True, path=path)
+    ref_o, ref_kv = orc.fwd_rec(q, k, v, lam.double().numpy(), want_state=True)
+    tol = TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4
+    assert_close(torch.cat([o1, o2], dim=2), ref_o, tol, "chained o")
+    assert_close(kv2, ref_kv, tol, "chained state")
+    assert_close(kv_full, ref_kv, tol, "one-call state")
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_decode_step_small(d, out_dtype):
+    B, H, S = 3, 5, 7
+    lam = inputs.decay_rates(5, 0.5)
+    gen = torch.Generator("cpu")
+    gen.manual_seed(9)
+    qs = inputs.draw((S, B, H, d), gen, "silu", torch.bfloat16)
+    ks = inputs.draw((S, B, H, d), gen, "silu", torch.bfloat16)
+    vs = inputs.draw((S, B, H, d), gen, "normal", torch.bfloat16)
+    kv0 = inputs.make_state(B, H, d, d, seed=10)
+    kv = kv0.to(DEV)
+    ref_kv = kv0.double().numpy().copy()
+    for s in range(S):
+        o = la.decode_step(qs[s].to(DEV), ks[s].to(DEV), vs[s].to(DEV), lam, kv, out_dtype=out_dtype)
+        ref = orc.decode_step(qs[s], ks[s], vs[s], lam.double().numpy(), ref_kv)
+        tol = 1e-5 if out_dtype == torch.float32 else 1e-2
+        assert_close(o.unsqueeze(2), ref[:, :, None, :], tol, "decode o")
+        assert_close(kv, ref_kv, 1e-5, "decode state")
+
+
+def test_decode_fp32_inputs():
+    B, H, d = 2, 2, 64
+    lam = torch.tensor([1.0, 0.5])
+    q, k, v, _ = inputs.make_qkvdo(B, H, 1, d, d, seed=11, dtype=torch.float32)
+    kv0 = inputs.make_state(B, H, d, d, seed=12)
+    kv = kv0.to(DEV)
+    ref_kv = kv0.double().numpy().copy()
+    o = la.decode_step(q[:, :, 0].contiguous().to(DEV), k[:, :, 0].contiguous().to(DEV),
+                       v[:, :, 0].contiguous().to(DEV), lam, kv)
+    ref = orc.decode_step(q[:, :, 0], k[:, :, 0], v[:, :, 0], lam.double().numpy(), ref_kv)
+    assert_close(o.unsqueeze(2), ref[:, :, None, :], 1e-5, "o")
+    assert_close(kv, ref_kv, 1e-6, "state")
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_bitwise_determinism(path):
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    q, k, v, do = inputs.make_qkvdo(1, 4, 1500, d, d, seed=13)
+    lam = inputs.decay_rates(4, 0.9)
+    a = fwd_bwd_gpu(q, k, v, do, lam, seg_len=256, path=path)
+    b = fwd_bwd_gpu(q, k, v, do, lam, seg_len=256, path=path)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_guard_bands_untouched(path):
+    """Outputs sit inside larger buffers filled with a sentinel; nothing outside the tensors may change."""
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N = 1, 3, 333
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=14)
+    lam = torch.tensor([1.0, 0.9, 0.5])
+    qg, kg, vg, dog = to_dev(q, k, v, do)
+    n = B * H * N * d
+    pad = 4096
+    sentinel = -1234.5
+    bufs = [torch.full((n + 2 * pad,), sentinel, dtype=torch.float32, device=DEV) for _ in range(4)]
+    views = [b[pad:pad + n].view(B, H, N, d) for b in bufs]
+    shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, 128, path)
+    la.la_fwd(shape, qg, kg, vg, lam, views[0], None, None, la.alloc_workspace(la.LA_OP_FWD, shape, DEV))
+    la.la_bwd(shape, qg, kg, vg, dog, lam, views[1], views[2], views[3], None, None, None,
+              la.alloc_workspace(la.LA_OP_BWD, shape, DEV))
+    torch.cuda.synchronize()
+    for b, vw in zip(bufs, views):
+        assert torch.all(b[:pad] == sentinel) and torch.all(b[pad + n:] == sentinel)
+        assert not torch.any(vw == sentinel)
+    ref = oracle_all(q, k, v, do, lam)
+    assert_close(views[0], ref[0], TOL_BF16, "o")
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_causality_bitwise(path):
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N, t0 = 1, 2, 400, 211
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=15)
+    lam = torch.tensor([1.0, 0.9])
+    q2, k2, v2, do2 = (x.clone() for x in (q, k, v, do))
+    q2[:, :, t0] += 1
+    k2[:, :, t0] -= 2
+    v2[:, :, t0] *= 3
+    a = fwd_bwd_gpu(q, k, v, do, lam, seg_len=128, path=path)
+    b = fwd_bwd_gpu(q2, k2, v2, do, lam, seg_len=128, path=path)
+    assert torch.equal(a[0][:, :, :t0], b[0][:, :, :t0])       # o
+    assert torch.equal(a[2][:, :, :t0], b[2][:, :, :t0])       # dq
+    do2[:, :, t0] += 1
+    c = fwd_bwd_gpu(q2, k, v, do2, lam, seg_len=128, path=path)
+    assert torch.equal(a[3][:, :, t0 + 1:], c[3][:, :, t0 + 1:])  # dk
+    assert torch.equal(a[4][:, :, t0 + 1:], c[4][:, :, t0 + 1:])  # dv
+
+
+def test_errors_on_device():
+    q, k, v, _ = inputs.make_qkvdo(1, 2, 64, 64, 64, seed=16)
+    qg, kg, vg = to_dev(q, k, v)
+    with pytest.raises(la.LaError):
+        la.fwd(qg, kg, vg, torch.tensor([1.0, 0.0]))
+    with pytest.raises(la.LaError):
+        la.fwd(qg, kg, vg, torch.tensor([1.0, 2.0]))
