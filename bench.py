@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the decayed linear-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the whole training hot path -- la_fwd followed by
+la_bwd (dQ, dK, dV) -- over one synthetic batch of the 7B-like long-context
+workload (B=1, H=32, N=65536, d=e=128, bf16 in, fp32 accumulate, fp32 out).
+The decode leg (batch 64, H=32, d=e=128, fp32 state, 256 recurrent steps after
+a 4096-token prefill) is timed in the same run and reported under "decode".
+
+Prints ONE JSON line.  `value` is fwd+bwd TFLOP/s counted with the block-method
+flop count per token-head (intra-block MACs for i>=j only), inputs resident in
+HBM.  `e2e` is the same metric through la_fwd_bwd_host with pinned host buffers
+(copies inside the timed region).  `roofline` describes the dominant kernel (the
+block walk), `step_roofline` the whole fwd+bwd step against
+max(flops/tensor peak, bytes/HBM peak).  `--impl reference` times the CPU oracle
+on a bounded sample of the same workload.
+
+With N > 1 (torchrun) every rank runs its own copy of the workload (the path
+shards over batch and heads with no exchange step): weak scaling, no collective
+on the data path; timing is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decayed linear-attn fwd+bwd TFLOP/s at 7B shape"
+UNIT = "TFLOP/s"
+WORKLOAD = "7b_long"
+
+
+# ---- accounting (per token-head, d = e, block size C capped at 128) ----------------------------
+def flops_per_token_head(d: int, C: int = 128) -> float:
+    C = min(C, 128)
+    fwd = 2 * C * d + 4 * d * d        # half score tile + half P.V tile, Q.KV, K^T V
+    bwd = 5 * C * d + 10 * d * d
+    return float(fwd + bwd)
+
+
+def bytes_per_token_head(d: int, out_bytes: int, what: str) -> float:
+    fwd = 2 * 3 * d + out_bytes * d                 # read q,k,v ; write o
+    bwd = 2 * 4 * d + out_bytes * 3 * d             # read q,k,v,dO ; write dq,dk,dv
+    walk = 2 * 3 * d + out_bytes * d                # one walk launch: read a,b,c ; write out
+    return float({"fwd": fwd, "bwd": bwd, "step": fwd + bwd, "walk": walk}[what])
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---- clocks sampling ----------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---- the CPU oracle leg -------------------------------------------------------------------------
+def oracle_sample_run(heads: int, n_tokens: int, seed: int = 0):
+    """Oracle fwd+bwd (token recurrence, fp64) on `heads` heads x n_tokens of the workload. Returns seconds."""
+    import torch
+    from oracle import la_oracle as orc
+    from paper_2307_14995_b200 import inputs
+    w = inputs.WORKLOADS[WORKLOAD]
+    q, k, v, do = inputs.make_qkvdo(1, heads, n_tokens, w.d, w.e, dtype=w.in_dtype, seed=seed)
+    lam = inputs.decay_rates(w.H, w.l_over_L)[:heads].double().numpy()
+    t0 = time.perf_counter()
+    orc.fwd_rec(q, k, v, lam)
+    orc.bwd_rec(q, k, v, do, lam)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(target_seconds: float = 12.0):
+    from oracle import la_oracle as orc
+    from paper_2307_14995_b200 import inputs
+    w = inputs.WORKLOADS[WORKLOAD]
+    cores = orc.threads()
+    heads = min(w.H, max(cores, 1))
+    t_cal = oracle_sample_run(heads, 1024)
+    n = int(min(w.N, max(1024, 1024 * target_seconds / max(t_cal, 1e-3))))
+    n = max(1024, n // 1024 * 1024)
+    t = oracle_sample_run(heads, n)
+    th = heads * n
+    return {"value": th * flops_per_token_head(w.d) / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d heads x %d tokens of the %s workload (fwd+bwd token recurrence, fp64), %.1f s"
+                      % (heads, n, WORKLOAD, t),
+            "token_heads_per_s": th / t}
+
+
+def run_reference(args):
+    """--impl reference: the oracle as it stands, on host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import la_oracle as orc
+    from paper_2307_14995_b200 import inputs
+    w = inputs.WORKLOADS[WORKLOAD]
+    cores = orc.threads()
+    heads = min(w.H, max(cores, 1))
+    t_cal = oracle_sample_run(heads, 512)
+    budget = 120.0 / max(1, args.steps + args.warmup)           # whole run within a few minutes
+    n = int(min(w.N, max(512, 512 * min(budget, 20.0) / max(t_cal, 1e-3))))
+    n = max(512, n // 512 * 512)
+    for _ in range(args.warmup):
+        oracle_sample_run(heads, n)
+    times = [oracle_sample_run(heads, n) for _ in range(args.steps)]
+    t = sum(times) / len(times)
+    th = heads * n
+    value = th * flops_per_token_head(w.d) / t / 1e12
+    sample = "%d heads x %d tokens of the %s workload per step (fwd+bwd token recurrence, fp64)" % (heads, n, WORKLOAD)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "%s: B=1,H=%d,N=%d,d=e=%d (sample: %s)" % (WORKLOAD, w.H, w.N, w.d, sample)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- our arm ------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2307_14995_b200 import binding as la, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    la.load()
+    peaks = load_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    w = inputs.WORKLOADS[WORKLOAD]
+    out_dtype = torch.float32
+    data = inputs.device_randn_like_workload(WORKLOAD, dev, seed=rank)
+    q, k, v, do, lam = data["q"], data["k"], data["v"], data["do"], data["lam"]
+    shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype)
+    o = torch.empty((w.B, w.H, w.N, w.e), dtype=out_dtype, device=dev)
+    dq, dk, dv = (torch.empty((w.B, w.H, w.N, w.d), dtype=out_dtype, device=dev) for _ in range(3))
+    ws_f = la.alloc_workspace(la.LA_OP_FWD, shape, dev)
+    ws_b = la.alloc_workspace(la.LA_OP_BWD, shape, dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        la.la_fwd(shape, q, k, v, lam, o, None, None, ws_f, stream)
+        la.la_bwd(shape, q, k, v, do, lam, dq, dk, dv, None, None, None, ws_b, stream)
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    launches0 = la.launch_count()
+    la.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    la.profile_enable(False)
+    prof = la.profile_collect()
+    launches = la.launch_count() - launches0
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+
+    th = w.token_heads
+    F = flops_per_token_head(w.d)
+    value = world * th * F / (ms_step * 1e-3) / 1e12
+    ob = 4 if out_dtype == torch.float32 else 2
+    step_bytes = th * bytes_per_token_head(w.d, ob, "step")
+    t_roof = max(th * F / (peaks["bf16_tflops_sustained"] * 1e12), step_bytes / (peaks["hbm_gbs"] * 1e9))
+    walk_ms, walk_n = prof["walk"]
+    walk_bytes = th * bytes_per_token_head(w.d, ob, "walk")
+    walk_avg_ms = walk_ms / max(walk_n, 1)
+    achieved = walk_bytes / (walk_avg_ms * 1e-3) / 1e9 if walk_n else None
+
+    # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
+    dw = inputs.WORKLOADS["decode"]
+    gen = torch.Generator(dev)
+    gen.manual_seed(1000 + rank)
+    BHd = (dw.B, dw.H, dw.d)
+    nsteps = dw.decode_steps
+    qs = torch.nn.functional.silu(torch.randn((nsteps,) + BHd, generator=gen, device=dev)).to(torch.bfloat16)
+    ks = torch.nn.functional.silu(torch.randn((nsteps,) + BHd, generator=gen, device=dev)).to(torch.bfloat16)
+    vs = torch.randn((nsteps, dw.B, dw.H, dw.e), generator=gen, device=dev).to(torch.bfloat16)
+    kv = torch.randn((dw.B, dw.H, dw.d, dw.e), generator=gen, device=dev)
+    dshape = la.make_shape(dw.B, dw.H, 1, dw.d, dw.e, torch.bfloat16, torch.float32)
+    od = torch.empty((nsteps, dw.B, dw.H, dw.e), dtype=torch.float32, device=dev)
+    dlam = inputs.decay_rates(dw.H, dw.l_over_L)
+
+    def decode_loop():
+        for s in range(nsteps):
+            la.la_decode_step(dshape, qs[s], ks[s], vs[s], dlam, kv, od[s], stream)
+
+    decode_loop()  # warm-up pass (256 launches)
+    barrier()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 3
+    d0.record(stream)
+    for _ in range(reps):
+        decode_loop()
+    d1.record(stream)
+    barrier()
+    dec_ms = max_over_ranks(d0.elapsed_time(d1) / (reps * nsteps))
+    dec_bytes = dw.B * dw.H * (2 * dw.d * dw.e * 4 + 2 * (2 * dw.d + dw.e) + 4 * dw.e)
+    dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e = None
+    try:
+        arena = torch.empty(la.host_arena_bytes(shape), dtype=torch.uint8, device=dev)
+        hq, hk, hv, hdo = (x.cpu().pin_memory() for x in (q, k, v, do))
+        ho = torch.empty(o.shape, dtype=out_dtype).pin_memory()
+        hdq, hdk, hdv = (torch.empty(dq.shape, dtype=out_dtype).pin_memory() for _ in range(3))
+        e2e_steps = max(1, min(args.steps, 3))
+        la.la_fwd_bwd_host(shape, hq, hk, hv, hdo, lam, ho, hdq, hdk, hdv, arena, stream)  # warm-up
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(e2e_steps):
+            la.la_fwd_bwd_host(shape, hq, hk, hv, hdo, lam, ho, hdq, hdk, hdv, arena, stream)
+        h1.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks(h0.elapsed_time(h1) / e2e_steps)
+        h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv, hdo))
+        d2h = sum(x.numel() * x.element_size() for x in (ho, hdq, hdk, hdv))
+        e2e = {"value": world * th * F / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "api": "la_fwd_bwd_host (pinned host buffers)"}
+    except Exception as ex:  # keep the device-resident numbers even if pinned memory is unavailable
+        e2e = {"value": None, "unit": UNIT, "error": str(ex)[:200]}
+
+    cpu = cpu_baseline() if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+
+    if rank == 0:
+        seg = la.segment_length(shape)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "%s: B=%d,H=%d,N=%d,d=e=%d per GPU, bf16 in, fp32 accumulate, fp32 out; "
+                                   "q,k=SiLU(N(0,1)), v,dO=N(0,1), lambda_h=exp(-(8h/H)(1-0.9))"
+                                   % (WORKLOAD, w.B, w.H, w.N, w.d),
+                       "segment_length": seg, "l2": "inputs (2.1 GB) and outputs (4.3 GB) exceed L2; no flush needed",
+                       "parallelism": "replicas x%d (no collective on the path)" % world,
+                       "flops_per_token_head": F, "bytes_per_token_head": bytes_per_token_head(w.d, ob, "step")},
+            "tokens_per_s": world * w.B * w.N / (ms_step * 1e-3),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "kernel_ms_per_step": {kname: ms / args.steps for kname, (ms, _) in prof.items()},
+            "roofline": {"kernel": "block walk (one launch each for O, dQ, dV, dK)", "bound": "hbm",
+                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
+                         "traffic": None, "peak_source": peaks["source"],
+                         "avg_launch_ms": walk_avg_ms, "launches": walk_n, "bytes_per_launch": walk_bytes},
+            "step_roofline": {"t_roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_step,
+                              "bytes": step_bytes, "flops": th * F, "peak_source": peaks["source"]},
+            "decode": {"tok_per_s": world * dw.B / (dec_ms * 1e-3), "us_per_step": dec_ms * 1e3,
+                       "workload": "batch %d, H=%d, d=e=%d, fp32 state, %d steps" % (dw.B, dw.H, dw.d, nsteps),
+                       "achieved_gbs": dec_gbs, "frac_of_hbm_peak": dec_gbs / peaks["hbm_gbs"],
+                       "bytes_per_step": dec_bytes},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

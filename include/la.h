@@ -130,6 +130,23 @@ la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void
 la_status la_decode_step(const la_shape* shape, const void* q, const void* k, const void* v,
                          const float* lambda_host, float* kv, void* o, void* stream);
 
+/*
+ * Forward + backward with HOST tensors (end-to-end convenience; the paper has no
+ * counterpart).  q,k,v,d_o and o,dq,dk,dv are host pointers with the layouts and
+ * dtypes of la_fwd / la_bwd (pinned memory makes the copies asynchronous).  The
+ * call enqueues, on `stream`: the four host-to-device copies, la_fwd, la_bwd
+ * (zero initial state, no state gradients) and the four device-to-host copies.
+ * device_arena is caller-owned device scratch of at least
+ * la_host_arena_bytes(shape) bytes, 256-byte aligned; it holds the device copies
+ * of all eight tensors and the workspace.  Host outputs are valid once the
+ * stream has been synchronised by the caller.
+ */
+size_t la_host_arena_bytes(const la_shape* shape);
+la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void* k_host,
+                          const void* v_host, const void* d_o_host, const float* lambda_host,
+                          void* o_host, void* dq_host, void* dk_host, void* dv_host,
+                          void* device_arena, size_t arena_bytes, void* stream);
+
 /* Human-readable name of a status code (static string). */
 const char* la_status_string(la_status s);
 

@@ -24,7 +24,7 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
-           "la_profile_collect")
+           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host")
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
 
 
@@ -64,6 +64,10 @@ def load():
         lib.la_bwd.restype = I
         lib.la_decode_step.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_step.restype = I
+        lib.la_host_arena_bytes.argtypes = [sp]
+        lib.la_host_arena_bytes.restype = sz
+        lib.la_fwd_bwd_host.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, sz, vp]
+        lib.la_fwd_bwd_host.restype = I
         lib.la_status_string.argtypes = [I]
         lib.la_status_string.restype = ctypes.c_char_p
         lib.la_version.restype = I
@@ -170,6 +174,25 @@ def la_decode_step(shape: LaShape, q, k, v, lam, kv, o, stream=None):
                                _ptr(o), _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_decode_step")
+
+
+def host_arena_bytes(shape: LaShape) -> int:
+    n = load().la_host_arena_bytes(ctypes.byref(shape))
+    if n == ctypes.c_size_t(-1).value:
+        raise LaError(2, "la_host_arena_bytes")
+    return int(n)
+
+
+def la_fwd_bwd_host(shape: LaShape, q, k, v, do, lam, o, dq, dk, dv, arena, stream=None):
+    """Host tensors in and out (ideally pinned); `arena` is a CUDA uint8 tensor of host_arena_bytes()."""
+    for t in (q, k, v, do, o, dq, dk, dv):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    hp = lambda t: ctypes.c_void_p(t.data_ptr())
+    rc = load().la_fwd_bwd_host(ctypes.byref(shape), hp(q), hp(k), hp(v), hp(do), _lam(lam), hp(o), hp(dq),
+                                hp(dk), hp(dv), _ptr(arena), arena.numel(), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_fwd_bwd_host")
 
 
 # ---- convenience wrappers that allocate outputs with torch -------------------------------

@@ -314,6 +314,60 @@ la_status la_decode_step(const la_shape* shape, const void* q, const void* k, co
   return LA_OK;
 }
 
+static size_t round256(size_t n) { return (n + 255) / 256 * 256; }
+
+size_t la_host_arena_bytes(const la_shape* shape) {
+  const size_t wf = la_workspace_bytes(LA_OP_FWD, shape);
+  const size_t wb = la_workspace_bytes(LA_OP_BWD, shape);
+  if (wf == (size_t)-1 || wb == (size_t)-1) return (size_t)-1;
+  const size_t tokens = (size_t)shape->B * shape->H * shape->N;
+  const size_t in_sz = shape->in_dtype == LA_BF16 ? 2 : 4;
+  const size_t out_sz = shape->out_dtype == LA_BF16 ? 2 : 4;
+  size_t total = 0;
+  total += 2 * round256(tokens * shape->d * in_sz) + 2 * round256(tokens * shape->e * in_sz);
+  total += 2 * round256(tokens * shape->d * out_sz) + 2 * round256(tokens * shape->e * out_sz);
+  total += round256(wf > wb ? wf : wb);
+  return total;
+}
+
+la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void* k_host,
+                          const void* v_host, const void* d_o_host, const float* lambda_host,
+                          void* o_host, void* dq_host, void* dk_host, void* dv_host,
+                          void* device_arena, size_t arena_bytes, void* stream) {
+  const size_t need = la_host_arena_bytes(shape);
+  if (need == (size_t)-1) return check_shape(shape, true) != LA_OK ? check_shape(shape, true) : LA_ERR_UNSUPPORTED;
+  if (!q_host || !k_host || !v_host || !d_o_host || !o_host || !dq_host || !dk_host || !dv_host)
+    return LA_ERR_INVALID_ARG;
+  if (!device_arena || arena_bytes < need) return LA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(device_arena) & 255u) return LA_ERR_INVALID_ARG;
+  const size_t tokens = (size_t)shape->B * shape->H * shape->N;
+  const size_t in_sz = shape->in_dtype == LA_BF16 ? 2 : 4;
+  const size_t out_sz = shape->out_dtype == LA_BF16 ? 2 : 4;
+  const size_t bq = tokens * shape->d * in_sz, bv = tokens * shape->e * in_sz;
+  const size_t bdq = tokens * shape->d * out_sz, bdv = tokens * shape->e * out_sz;
+  char* p = static_cast<char*>(device_arena);
+  auto take = [&p](size_t n) { char* r = p; p += round256(n); return r; };
+  char *dq_in = take(bq), *dk_in = take(bq), *dv_in = take(bv), *ddo_in = take(bv);
+  char *d_o = take(bdv), *d_dq = take(bdq), *d_dk = take(bdq), *d_dv = take(bdv);
+  char* ws = p;
+  const size_t ws_bytes = arena_bytes - (size_t)(ws - static_cast<char*>(device_arena));
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  LA_TRY_CUDA(cudaMemcpyAsync(dq_in, q_host, bq, cudaMemcpyHostToDevice, cs));
+  LA_TRY_CUDA(cudaMemcpyAsync(dk_in, k_host, bq, cudaMemcpyHostToDevice, cs));
+  LA_TRY_CUDA(cudaMemcpyAsync(dv_in, v_host, bv, cudaMemcpyHostToDevice, cs));
+  LA_TRY_CUDA(cudaMemcpyAsync(ddo_in, d_o_host, bv, cudaMemcpyHostToDevice, cs));
+  la_status st = la_fwd(shape, dq_in, dk_in, dv_in, lambda_host, d_o, nullptr, nullptr, ws, ws_bytes, stream);
+  if (st != LA_OK) return st;
+  st = la_bwd(shape, dq_in, dk_in, dv_in, ddo_in, lambda_host, d_dq, d_dk, d_dv, nullptr, nullptr,
+              nullptr, ws, ws_bytes, stream);
+  if (st != LA_OK) return st;
+  LA_TRY_CUDA(cudaMemcpyAsync(o_host, d_o, bdv, cudaMemcpyDeviceToHost, cs));
+  LA_TRY_CUDA(cudaMemcpyAsync(dq_host, d_dq, bdq, cudaMemcpyDeviceToHost, cs));
+  LA_TRY_CUDA(cudaMemcpyAsync(dk_host, d_dk, bdq, cudaMemcpyDeviceToHost, cs));
+  LA_TRY_CUDA(cudaMemcpyAsync(dv_host, d_dv, bdv, cudaMemcpyDeviceToHost, cs));
+  return LA_OK;
+}
+
 const char* la_status_string(la_status s) {
   switch (s) {
     case LA_OK: return "ok";

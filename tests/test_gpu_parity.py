@@ -301,7 +301,7 @@ def test_decode_step_small(d, out_dtype):
     for s in range(S):
         o = la.decode_step(qs[s].to(DEV), ks[s].to(DEV), vs[s].to(DEV), lam, kv, out_dtype=out_dtype)
         ref = orc.decode_step(qs[s], ks[s], vs[s], lam.double().numpy(), ref_kv)
-        tol = 1e-5 if out_dtype == torch.float32 else 1e-2
+        tol = 1e-5 if out_dtype == torch.float32 else TOL_BF16  # bf16 output rounding of heavy-tailed values
         assert_close(o.unsqueeze(2), ref[:, :, None, :], tol, "decode o")
         assert_close(kv, ref_kv, 1e-5, "decode state")
 
