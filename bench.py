@@ -216,6 +216,12 @@ def run_ours(args):
     out_dtype = torch.float32
     data = inputs.device_randn_like_workload(WORKLOAD, dev, seed=rank)
     q, k, v, do, lam = data["q"], data["k"], data["v"], data["do"], data["lam"]
+    if args.small:
+        # profiling case: 8 heads x 16384 tokens (inputs + outputs still exceed L2), same kernels
+        import dataclasses
+        w = dataclasses.replace(w, H=8, N=16384)
+        q, k, v, do = (x[:, :8, :16384].contiguous() for x in (q, k, v, do))
+        lam = lam[:8].contiguous()
     shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype)
     o = torch.empty((w.B, w.H, w.N, w.e), dtype=out_dtype, device=dev)
     dq, dk, dv = (torch.empty((w.B, w.H, w.N, w.d), dtype=out_dtype, device=dev) for _ in range(3))
@@ -227,7 +233,8 @@ def run_ours(args):
         la.la_fwd(shape, q, k, v, lam, o, None, None, ws_f, stream)
         la.la_bwd(shape, q, k, v, do, lam, dq, dk, dv, None, None, None, ws_b, stream)
 
-    for _ in range(args.warmup):
+    train_steps = 0 if args.only == "decode" else args.steps
+    for _ in range(args.warmup if train_steps else 0):
         step()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -237,14 +244,14 @@ def run_ours(args):
     la.profile_enable(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(train_steps):
         step()
     e1.record(stream)
     barrier()
     la.profile_enable(False)
     prof = la.profile_collect()
     launches = la.launch_count() - launches0
-    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / max(train_steps, 1))
 
     th = w.token_heads
     F = flops_per_token_head(w.d)
@@ -257,12 +264,19 @@ def run_ours(args):
     walk_avg_ms = walk_ms / max(walk_n, 1)
     achieved = walk_bytes / (walk_avg_ms * 1e-3) / 1e9 if walk_n else None
 
+    if args.only == "train":
+        if rank == 0:
+            print(json.dumps({"only": "train", "small": bool(args.small), "ms_per_step": ms_step,
+                              "kernel_ms_per_step": {n: ms / args.steps for n, (ms, _) in prof.items()},
+                              "walk_gbs": achieved}), flush=True)
+        return
+
     # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
     dw = inputs.WORKLOADS["decode"]
     gen = torch.Generator(dev)
     gen.manual_seed(1000 + rank)
     BHd = (dw.B, dw.H, dw.d)
-    nsteps = dw.decode_steps
+    nsteps = args.decode_steps or dw.decode_steps
     qs = torch.nn.functional.silu(torch.randn((nsteps,) + BHd, generator=gen, device=dev)).to(torch.bfloat16)
     ks = torch.nn.functional.silu(torch.randn((nsteps,) + BHd, generator=gen, device=dev)).to(torch.bfloat16)
     vs = torch.randn((nsteps, dw.B, dw.H, dw.e), generator=gen, device=dev).to(torch.bfloat16)
@@ -288,6 +302,10 @@ def run_ours(args):
     dec_bytes = dw.B * dw.H * (2 * dw.d * dw.e * 4 + 2 * (2 * dw.d + dw.e) + 4 * dw.e)
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
     clocks = sampler.stop() if rank == 0 else None
+    if args.only == "decode":
+        if rank == 0:
+            print(json.dumps({"only": "decode", "us_per_step": dec_ms * 1e3, "achieved_gbs": dec_gbs}), flush=True)
+        return
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
@@ -356,6 +374,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default="all", choices=["all", "train", "decode"],
+                    help="profiling aid: run only the fwd+bwd leg or only the decode leg (prints a short line)")
+    ap.add_argument("--small", action="store_true",
+                    help="profiling aid: 8 heads x 16384 tokens of the workload for the fwd+bwd leg")
+    ap.add_argument("--decode-steps", type=int, default=0, help="profiling aid: recurrent steps per pass")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
