@@ -50,7 +50,7 @@ typedef enum {
   LA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than la_workspace_bytes() */
   LA_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed */
   LA_ERR_ARCH = 5,        /* current device is not sm_100 */
-  LA_ERR_DEVICE_TIMEOUT = 6 /* a bounded device-side wait expired (see la_read_device_status) */
+  LA_ERR_DEVICE_TIMEOUT = 6 /* a bounded device-side wait expired (see la_device_status) */
 } la_status;
 
 typedef enum { LA_BF16 = 0, LA_F32 = 1 } la_dtype;
@@ -146,6 +146,16 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
                           const void* v_host, const void* d_o_host, const float* lambda_host,
                           void* o_host, void* dq_host, void* dk_host, void* dv_host,
                           void* device_arena, size_t arena_bytes, void* stream);
+
+/*
+ * Device-side failure flag (no counterpart in the paper).  The tensor-core kernels
+ * never spin without limit: a thread block whose wait on a copy or on the tensor
+ * cores expires records a code, drains what it started and returns, leaving its
+ * part of the output unwritten.  This call copies the flag back (it blocks until
+ * the device is idle), stores the raw code in *code if code is not NULL, clears
+ * the flag, and returns LA_OK if no block failed, else LA_ERR_DEVICE_TIMEOUT.
+ */
+la_status la_device_status(unsigned int* code);
 
 /* Human-readable name of a status code (static string). */
 const char* la_status_string(la_status s);

@@ -24,7 +24,7 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
-           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host")
+           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status")
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
 
 
@@ -68,6 +68,8 @@ def load():
         lib.la_host_arena_bytes.restype = sz
         lib.la_fwd_bwd_host.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, sz, vp]
         lib.la_fwd_bwd_host.restype = I
+        lib.la_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
+        lib.la_device_status.restype = I
         lib.la_status_string.argtypes = [I]
         lib.la_status_string.restype = ctypes.c_char_p
         lib.la_version.restype = I
@@ -91,6 +93,15 @@ def version() -> int:
 
 def launch_count() -> int:
     return int(load().la_launch_count())
+
+
+def device_status() -> int:
+    """Blocks until the device is idle; raises if a tensor-core block gave up on a bounded wait."""
+    code = ctypes.c_uint(0)
+    rc = load().la_device_status(ctypes.byref(code))
+    if rc != 0:
+        raise LaError(rc, "la_device_status (device code %d)" % code.value)
+    return int(code.value)
 
 
 def profile_enable(on: bool) -> None:

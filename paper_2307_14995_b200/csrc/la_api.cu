@@ -368,6 +368,14 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
   return LA_OK;
 }
 
+la_status la_device_status(unsigned int* code) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return LA_ERR_CUDA;
+  const unsigned int v = tc_read_status(true);
+  if (code) *code = v;
+  if (v == 0xFFFFFFFFu) return LA_ERR_CUDA;
+  return v == 0 ? LA_OK : LA_ERR_DEVICE_TIMEOUT;
+}
+
 const char* la_status_string(la_status s) {
   switch (s) {
     case LA_OK: return "ok";

@@ -78,6 +78,10 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int out_dt
 cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int precision,
                               cudaStream_t stream);
 
+// Failure code recorded by a tensor-core block whose bounded wait expired (0 = none);
+// copies it from the device (blocking) and optionally clears it.
+unsigned int tc_read_status(bool clear);
+
 void count_launch(int n = 1);
 
 // Brackets one kernel launch with CUDA events when benchmark profiling is enabled
