@@ -96,6 +96,7 @@ la_status make_plan(const la_shape* s, Plan* p) {
   }
   p->seg_len = (int)seg_len;
   p->nseg = (int)((s->N + seg_len - 1) / seg_len);
+  if (p->nseg > 1024) return LA_ERR_UNSUPPORTED;  // the state scan keeps one decay factor per segment on chip
   return LA_OK;
 }
 

@@ -282,29 +282,53 @@ simt_prepass_kernel(const OpArgs args, const DecayTable tab) {
 // Turns segment-local states into the state entering each segment, in place:
 //   forward: x_0 = Z_in, x_{p+1} = lambda^(L_p) x_p + local_p
 //   reverse: x_{last} = Z_in, x_{p-1} = lambda^(L_p) x_p + local_p
-// One thread per state element; the walk over segments is sequential and short.
-__global__ void scan_kernel(const ScanArgs args, const DecayTable tab) {
-  const int DE = args.Da * args.Ec;
-  const long total = (long)args.BH * DE;
-  const long gid = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (gid >= total) return;
-  const int bh = (int)(gid / DE);
-  const int idx = (int)(gid % DE);
-  const int x = idx / args.Ec, y = idx % args.Ec;
-  const int idx_t = y * args.Da + x;
+// One thread block per 32x32 tile of one (batch*head) state; each thread carries four elements
+// across the short sequential walk over segments.  The optional transposed copy goes through a
+// shared-memory tile so that both copies are written with coalesced stores.
+constexpr int SCAN_MAX_SEG = 1024;
+__global__ void __launch_bounds__(256) scan_kernel(const ScanArgs args, const DecayTable tab) {
+  __shared__ float gamma[SCAN_MAX_SEG];
+  __shared__ float tile[32][33];
+  const int Da = args.Da, Ec = args.Ec, DE = Da * Ec;
+  const int bh = blockIdx.x;
+  const int tiles_y = Ec / 32;
+  const int x0 = (blockIdx.y / tiles_y) * 32, y0 = (blockIdx.y % tiles_y) * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
   const double s2 = tab.s2[bh % args.H];
-  float z = 0.f;
-  if (args.z_in) z = args.z_in[(size_t)bh * DE + (args.z_in_transposed ? idx_t : idx)];
+  for (int p = threadIdx.x; p < args.nseg; p += 256) {
+    const int L = min(args.N, (p + 1) * args.seg_len) - p * args.seg_len;
+    gamma[p] = decay_pow_d(s2, (double)L);
+  }
+  float z[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int x = x0 + ty + 8 * k, y = y0 + tx;
+    z[k] = 0.f;
+    if (args.z_in) z[k] = args.z_in[(size_t)bh * DE + (args.z_in_transposed ? (y * Da + x) : (x * Ec + y))];
+  }
+  __syncthreads();
   for (int ip = 0; ip < args.nseg; ++ip) {
     const int p = args.reverse ? (args.nseg - 1 - ip) : ip;
     const size_t off = ((size_t)bh * args.nseg + p) * DE;
     const bool more = (ip + 1 < args.nseg);
-    const float loc = more ? args.buf[off + idx] : 0.f;
-    args.buf[off + idx] = z;
-    if (args.buf_t) args.buf_t[off + idx_t] = z;
+    float loc[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) loc[k] = more ? args.buf[off + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] : 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) args.buf[off + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] = z[k];
+    if (args.buf_t) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) tile[ty + 8 * k][tx] = z[k];
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        args.buf_t[off + (size_t)(y0 + ty + 8 * k) * Da + x0 + tx] = tile[tx][ty + 8 * k];
+      __syncthreads();
+    }
     if (more) {
-      const int L = min(args.N, (p + 1) * args.seg_len) - p * args.seg_len;
-      z = fmaf(decay_pow_d(s2, (double)L), z, loc);
+      const float g = gamma[p];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) z[k] = fmaf(g, z[k], loc[k]);
     }
   }
 }
@@ -385,11 +409,10 @@ cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int D
 }
 
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream) {
-  const long total = (long)args.BH * args.Da * args.Ec;
-  const int block = 256;
-  const unsigned grid = (unsigned)((total + block - 1) / block);
+  if (args.nseg > SCAN_MAX_SEG || (args.Da % 32) != 0 || (args.Ec % 32) != 0) return cudaErrorInvalidValue;
+  const dim3 grid((unsigned)args.BH, (unsigned)((args.Da / 32) * (args.Ec / 32)));
   KernelTimer timer(K_SCAN, stream);
-  scan_kernel<<<grid, block, 0, stream>>>(args, tab);
+  scan_kernel<<<grid, 256, 0, stream>>>(args, tab);
   count_launch();
   return cudaGetLastError();
 }
