@@ -50,7 +50,8 @@ typedef enum {
   LA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than la_workspace_bytes() */
   LA_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed */
   LA_ERR_ARCH = 5,        /* current device is not sm_100 */
-  LA_ERR_DEVICE_TIMEOUT = 6 /* a bounded device-side wait expired (see la_device_status) */
+  LA_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait expired (see la_device_status) */
+  LA_ERR_SCRATCH_LIMIT = 7   /* la_fwd_noalloc: the shape needs more scratch than the built-in buffer holds */
 } la_status;
 
 typedef enum { LA_BF16 = 0, LA_F32 = 1 } la_dtype;
@@ -129,6 +130,30 @@ la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void
  */
 la_status la_decode_step(const la_shape* shape, const void* q, const void* k, const void* v,
                          const float* lambda_host, float* kv, void* o, void* stream);
+
+/*
+ * Forward pass without caller-provided scratch (the paper has no counterpart; this is a
+ * deployment convenience).  Same result as la_fwd, but the per-segment state scratch comes
+ * from a fixed LA_NOALLOC_SCRATCH_BYTES array that is part of the library's device image,
+ * for callers that cannot allocate device memory when they call: a server that gave all
+ * device memory to its own pool at start-up, a latency-critical loop that must avoid the
+ * device-wide synchronisation of an allocation, or a plug-in that is handed only tensor
+ * pointers and a stream.  Inputs and outputs are still the caller's.
+ *   - Every GPU that loads the library holds the 32 MiB array until the process exits.
+ *   - Shapes with la_workspace_bytes(LA_OP_FWD, shape) > LA_NOALLOC_SCRATCH_BYTES are
+ *     rejected with LA_ERR_SCRATCH_LIMIT before anything is launched.
+ *   - The first call on each device looks up the array's device address (once, with that
+ *     device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the array: calls that can overlap on the GPU (different
+ *     streams) race on it; calls ordered on one stream are safe.  The array keeps the last
+ *     call's contents, which needs no clearing: the forward pass writes every scratch
+ *     element before reading it.
+ * The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ */
+#define LA_NOALLOC_SCRATCH_BYTES (32u << 20)
+la_status la_fwd_noalloc(const la_shape* shape, const void* q, const void* k, const void* v,
+                         const float* lambda_host, void* o, const float* kv_in, float* kv_out,
+                         void* stream);
 
 /*
  * Forward + backward with HOST tensors (end-to-end convenience; the paper has no

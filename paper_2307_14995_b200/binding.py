@@ -24,7 +24,8 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
-           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status")
+           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc")
+LA_NOALLOC_SCRATCH_BYTES = 32 << 20
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
 
 
@@ -60,6 +61,8 @@ def load():
         lib.la_segment_length.restype = I
         lib.la_fwd.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp, vp, sz, vp]
         lib.la_fwd.restype = I
+        lib.la_fwd_noalloc.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp, vp]
+        lib.la_fwd_noalloc.restype = I
         lib.la_bwd.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.la_bwd.restype = I
         lib.la_decode_step.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
@@ -168,6 +171,17 @@ def la_fwd(shape: LaShape, q, k, v, lam, o, kv_in=None, kv_out=None, workspace=N
                        _ptr(kv_out), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_fwd")
+
+
+def la_fwd_noalloc(shape: LaShape, q, k, v, lam, o, kv_in=None, kv_out=None, stream=None):
+    """la_fwd with the library's built-in static scratch: for callers that cannot allocate device
+    memory when they call (everything was handed to a pool at start-up, no allocator is available,
+    or an allocation's device-wide synchronisation is unacceptable).  Calls on different streams
+    must not overlap; shapes needing more than LA_NOALLOC_SCRATCH_BYTES raise LaError (status 7)."""
+    rc = load().la_fwd_noalloc(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(o), _ptr(kv_in),
+                               _ptr(kv_out), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_fwd_noalloc")
 
 
 def la_bwd(shape: LaShape, q, k, v, do, lam, dq, dk, dv, kv_in=None, grad_kv_out=None, grad_kv_in=None,

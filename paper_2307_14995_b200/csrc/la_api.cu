@@ -386,6 +386,7 @@ const char* la_status_string(la_status s) {
     case LA_ERR_CUDA: return "CUDA call or launch failed";
     case LA_ERR_ARCH: return "device is not sm_100";
     case LA_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+    case LA_ERR_SCRATCH_LIMIT: return "shape needs more scratch than the built-in static buffer holds";
   }
   return "unknown status";
 }
