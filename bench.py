@@ -80,7 +80,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -234,11 +234,12 @@ def run_ours(args):
         la.la_bwd(shape, q, k, v, do, lam, dq, dk, dv, None, None, None, ws_b, stream)
 
     train_steps = 0 if args.only == "decode" else args.steps
-    for _ in range(args.warmup if train_steps else 0):
-        step()
+    # clocks are sampled from before the warm-up until the last timed leg has finished
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+    for _ in range(args.warmup if train_steps else 0):
+        step()
     barrier()
     launches0 = la.launch_count()
     la.profile_enable(True)
@@ -266,7 +267,7 @@ def run_ours(args):
 
     if args.only == "train":
         if rank == 0:
-            print(json.dumps({"only": "train", "small": bool(args.small), "ms_per_step": ms_step,
+            print(json.dumps({"only": "train", "small": bool(args.small), "ms_per_step": ms_step, "clocks": sampler.stop(),
                               "kernel_ms_per_step": {n: ms / args.steps for n, (ms, _) in prof.items()},
                               "walk_gbs": achieved}), flush=True)
         return
@@ -301,7 +302,7 @@ def run_ours(args):
     dec_ms = max_over_ranks(d0.elapsed_time(d1) / (reps * nsteps))
     dec_bytes = dw.B * dw.H * (2 * dw.d * dw.e * 4 + 2 * (2 * dw.d + dw.e) + 4 * dw.e)
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = None
     if args.only == "decode":
         if rank == 0:
             print(json.dumps({"only": "decode", "us_per_step": dec_ms * 1e3, "achieved_gbs": dec_gbs}), flush=True)
@@ -332,6 +333,7 @@ def run_ours(args):
     except Exception as ex:  # keep the device-resident numbers even if pinned memory is unavailable
         e2e = {"value": None, "unit": UNIT, "error": str(ex)[:200]}
 
+    clocks = sampler.stop() if rank == 0 else None
     cpu = cpu_baseline() if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
 
     if rank == 0:

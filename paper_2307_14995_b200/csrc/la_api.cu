@@ -82,17 +82,27 @@ la_status make_plan(const la_shape* s, Plan* p) {
                      : s->precision;
   long seg_len = s->seg_len;
   if (seg_len == 0) {
-    // Enough independent thread blocks to cover the 148 SMs a few times over, but
-    // segments no shorter than 1024 tokens so the per-segment state traffic stays small.
-    const long target = 592;
+    // One thread block per (batch*head, segment[, value-column half]) and one block per SM at a
+    // time: pick the segment count that minimises (waves over the 148 SMs) x (blocks walked per
+    // segment + pipeline fill), with segments no shorter than 1024 tokens so that the
+    // per-segment state traffic stays small.  Depends on the shape only.
     const long slices = p->tensor ? 2 : 1;  // the tensor kernels also split the value columns
-    long want = (target + p->BH * slices - 1) / (p->BH * slices);
+    const long sms = 148, fill = 2;
     long most = s->N / 1024;
     if (most < 1) most = 1;
-    if (want > most) want = most;
-    if (want < 1) want = 1;
-    seg_len = (s->N + want - 1) / want;
-    seg_len = (seg_len + 127) / 128 * 128;
+    if (most > 1024) most = 1024;
+    long best_n = 1, best_cost = -1;
+    for (long n = 1; n <= most; ++n) {
+      const long len = ((s->N + n - 1) / n + 127) / 128 * 128;
+      const long nseg = (s->N + len - 1) / len;
+      const long waves = (p->BH * slices * nseg + sms - 1) / sms;
+      const long cost = waves * (len / 128 + fill);
+      if (best_cost < 0 || cost < best_cost) {
+        best_cost = cost;
+        best_n = n;
+      }
+    }
+    seg_len = ((s->N + best_n - 1) / best_n + 127) / 128 * 128;
   }
   p->seg_len = (int)seg_len;
   p->nseg = (int)((s->N + seg_len - 1) / seg_len);

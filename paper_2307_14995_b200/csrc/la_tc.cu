@@ -89,6 +89,7 @@ struct alignas(1024) TcSmem {
 };
 
 struct TcArgs {
+  const void* c;  // value-like tensor, also read row-wise straight from global memory by the Z group
   void* out;
   const float* entry;
   float* local_out;
@@ -100,12 +101,11 @@ struct TcArgs {
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  unsigned spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 31u) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_BUDGET) return false;
-    }
+  // each try may sleep in hardware for up to 20 us; a polling warp would otherwise take issue
+  // slots from the warps that share its scheduler
+  while (!mbar_try_wait_hint(bar, parity, 20000u)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_BUDGET) return false;
   }
   return true;
 }
@@ -149,10 +149,21 @@ __device__ __forceinline__ void store_pairs16(__nv_bfloat16* tile, int row, int 
 __device__ long long* g_tc_trace = nullptr;
 #define TC_TRACE(it, ev)                                                                          \
   do {                                                                                            \
-    if (g_tc_trace && blockIdx.x == 0 && (it) < 64) g_tc_trace[(it) * 32 + (ev)] = clock64();     \
+    if (g_tc_trace && blockIdx.x == 270 && (it) < 64) g_tc_trace[(it) * 32 + (ev)] = clock64();     \
+  } while (0)
+__device__ unsigned long long* g_tc_cta_times = nullptr;  // [grid][2] start/end in ns (walk kernels only)
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define TC_CTA_TIME(slot)                                                                          \
+  do {                                                                                             \
+    if (!STATE_ONLY && g_tc_cta_times && threadIdx.x == 0) g_tc_cta_times[blockIdx.x * 2 + (slot)] = globaltimer_ns(); \
   } while (0)
 #else
 #define TC_TRACE(it, ev) do { } while (0)
+#define TC_CTA_TIME(slot) do { } while (0)
 #endif
 
 #define TC_WAIT(barid, par, code)                                        \
@@ -208,6 +219,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_slot;
+  TC_CTA_TIME(0);
   bool issued_mma = false;
   int armed_a[2] = {0, 0}, armed_b[2] = {0, 0}, armed_c[2] = {0, 0};  // producer: uses armed per stage
 
@@ -420,25 +432,24 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     const int r = q * 32 + lane;      // token row j of c / state row k of Z
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
 
-    // fc = diag(f_state) c for block iteration `it` (this warp's 32 columns), into the buffer at hi_tile / lo_tile
-    auto make_fc = [&](int it, __nv_bfloat16* hi_tile, __nv_bfloat16* lo_tile) {
+    // Decay factor of row r of block iteration `it` in the state update.
+    auto state_factor = [&](int it) -> float {
       const int blk = REV ? (nblk - 1 - it) : it;
       const int t0 = seg_t0 + blk * 128;
       const int Cr = min(128, seg_t1 - t0);
-      float f = 0.f;
-      if (r < Cr) {
-        if (STATE_ONLY)
-          f = REV ? exp2f(-s2 * (float)(t0 + r - seg_t0 + 1)) : exp2f(-s2 * (float)(seg_t1 - 1 - t0 - r));
-        else
-          f = REV ? exp2f(-s2 * (float)(r + 1)) : exp2f(-s2 * (float)(Cr - 1 - r));
-      }
-      const __nv_bfloat16* ctile = &sm.st[it & 1].c[0];
+      if (r >= Cr) return 0.f;
+      if (STATE_ONLY)
+        return REV ? exp2f(-s2 * (float)(t0 + r - seg_t0 + 1)) : exp2f(-s2 * (float)(seg_t1 - 1 - t0 - r));
+      return REV ? exp2f(-s2 * (float)(r + 1)) : exp2f(-s2 * (float)(Cr - 1 - r));
+    };
+    // fc = diag(f_state) c for this warp's 32 columns of row r, given as 4 x 8 raw bf16 (chunks
+    // 4*zh .. 4*zh+3 of the 64-column row), into the swizzled operand buffer at hi_tile / lo_tile.
+    auto make_fc = [&](const uint4 (&raw)[4], float f, __nv_bfloat16* hi_tile, __nv_bfloat16* lo_tile) {
 #pragma unroll
       for (int gg = 0; gg < 2; ++gg) {  // 16 elements per pass
         const int g = zh * 2 + gg;
-        const uint4 raw0 = *reinterpret_cast<const uint4*>(ctile + r * 64 + (((2 * g) ^ (r & 7)) << 3));
-        const uint4 raw1 = *reinterpret_cast<const uint4*>(ctile + r * 64 + (((2 * g + 1) ^ (r & 7)) << 3));
-        const uint32_t w[8] = {raw0.x, raw0.y, raw0.z, raw0.w, raw1.x, raw1.y, raw1.z, raw1.w};
+        const uint32_t w[8] = {raw[2 * gg].x, raw[2 * gg].y, raw[2 * gg].z, raw[2 * gg].w,
+                               raw[2 * gg + 1].x, raw[2 * gg + 1].y, raw[2 * gg + 1].z, raw[2 * gg + 1].w};
         float x16[16];
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
@@ -453,13 +464,37 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       }
       fence_proxy_async_smem();
     };
+    // this thread's row slice of the c tile in shared memory (state-only kernel)
+    auto c_from_tile = [&](int it, uint4 (&raw)[4]) {
+      const __nv_bfloat16* ctile = &sm.st[it & 1].c[0];
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+        raw[x] = *reinterpret_cast<const uint4*>(ctile + r * 64 + (((4 * zh + x) ^ (r & 7)) << 3));
+    };
+    // the same slice straight from global memory (walk kernel: keeps the shared c tile off the state
+    // chain, so that tile only has to arrive in time for M4); rows beyond N read as zero
+    auto c_from_global = [&](int it, uint4 (&raw)[4]) {
+      const int blk = REV ? (nblk - 1 - it) : it;
+      const int t = seg_t0 + blk * 128 + r;
+      if (t < args.N) {
+        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(args.c) +
+                                                          ((size_t)bh * args.N + t) * 128 + ehalf * 64 + zh * 32);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) raw[x] = __ldg(src + x);
+      } else {
+#pragma unroll
+        for (int x = 0; x < 4; ++x) raw[x] = make_uint4(0u, 0u, 0u, 0u);
+      }
+    };
 
     if (STATE_ONLY) {
       for (int it = 0; it < nblk; ++it) {
         const int s = it & 1;
         TC_WAIT(FULL_C0 + s, (it >> 1) & 1, 18);
         if (it >= 2) TC_WAIT(FC_FREE0 + s, ((it >> 1) - 1) & 1, 19);  // the MMA two blocks back has read this buffer
-        make_fc(it, s ? sm.z_hi : sm.fc_hi, s ? sm.z_lo : sm.fc_lo);
+        uint4 craw[4];
+        c_from_tile(it, craw);
+        make_fc(craw, state_factor(it), s ? sm.z_hi : sm.fc_hi, s ? sm.z_lo : sm.fc_lo);
         mbar_arrive(&sm.bars[FC_READY0 + s]);
         mbar_arrive(&sm.bars[C_FREE0 + s]);
       }
@@ -514,9 +549,11 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       };
       write_state_operand();
       mbar_arrive(&sm.bars[Z_READY]);
-      TC_WAIT(FULL_C0, 0, 21);
-      make_fc(0, sm.fc_hi, sm.fc_lo);
+      uint4 cnext[4];  // row slice of the next block's c, fetched one block ahead
+      c_from_global(0, cnext);
+      make_fc(cnext, state_factor(0), sm.fc_hi, sm.fc_lo);
       mbar_arrive(&sm.bars[FC_READY0]);
+      if (nblk > 1) c_from_global(1, cnext);
 
       for (int it = 0; it < nblk; ++it) {
         const int blk = REV ? (nblk - 1 - it) : it;
@@ -545,9 +582,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
         if (it + 1 < nblk) {
           // DZ_READY also says M3 of this block is done, so the fc buffer may be rewritten
-          TC_WAIT(FULL_C0 + ((it + 1) & 1), ((it + 1) >> 1) & 1, 24);
-          make_fc(it + 1, sm.fc_hi, sm.fc_lo);
+          make_fc(cnext, state_factor(it + 1), sm.fc_hi, sm.fc_lo);
           mbar_arrive(&sm.bars[FC_READY0]);
+          if (it + 2 < nblk) c_from_global(it + 2, cnext);
           if (tid == 384) TC_TRACE(it, 10);
           // Z_FREE: M2 of this block has read the old state operand
           TC_WAIT(Z_FREE, it & 1, 23);
@@ -656,6 +693,7 @@ teardown:
   }
   tc_fence_before_sync();
   __syncthreads();
+  TC_CTA_TIME(1);
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
@@ -713,7 +751,7 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int out_dt
   if (!make_map(&ma, args.a, args.N, args.BH) || !make_map(&mb, args.b, args.N, args.BH) ||
       !make_map(&mc, args.c, args.N, args.BH))
     return cudaErrorInvalidValue;
-  TcArgs ta{args.out, args.entry, nullptr, args.final_out, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
+  TcArgs ta{args.c, args.out, args.entry, nullptr, args.final_out, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
   if (args.reverse)
     return f32 ? launch_t<true, false, float>(ma, mb, mc, ta, tab, stream)
                : launch_t<true, false, __nv_bfloat16>(ma, mb, mc, ta, tab, stream);
@@ -725,7 +763,7 @@ cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int pre
   CUtensorMap mb, mc;
   if (!make_map(&mb, args.b, args.N, args.BH) || !make_map(&mc, args.c, args.N, args.BH))
     return cudaErrorInvalidValue;
-  TcArgs ta{nullptr, nullptr, args.local_out, nullptr, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
+  TcArgs ta{args.c, nullptr, nullptr, args.local_out, nullptr, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
   // the a map is unused by the state-only kernel; pass a valid descriptor anyway
   return args.reverse ? launch_t<true, true, float>(mb, mb, mc, ta, tab, stream)
                       : launch_t<false, true, float>(mb, mb, mc, ta, tab, stream);
@@ -734,6 +772,9 @@ cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int pre
 #ifdef LA_TC_TRACE
 extern "C" void la_debug_set_trace(long long* device_buffer) {
   cudaMemcpyToSymbol(g_tc_trace, &device_buffer, sizeof(device_buffer));
+}
+extern "C" void la_debug_set_cta_times(unsigned long long* device_buffer) {
+  cudaMemcpyToSymbol(g_tc_cta_times, &device_buffer, sizeof(device_buffer));
 }
 #endif
 
