@@ -307,13 +307,23 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs args, const De
     if (args.z_in) z[k] = args.z_in[(size_t)bh * DE + (args.z_in_transposed ? (y * Da + x) : (x * Ec + y))];
   }
   __syncthreads();
+  // the local state of a segment is fetched one step ahead of its use: the chain over segments is
+  // sequential, and this keeps one global-memory round trip out of every step
+  auto seg_of = [&](int ip) { return args.reverse ? (args.nseg - 1 - ip) : ip; };
+  float loc[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    loc[k] = (args.nseg > 1) ? args.buf[((size_t)bh * args.nseg + seg_of(0)) * DE + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] : 0.f;
   for (int ip = 0; ip < args.nseg; ++ip) {
-    const int p = args.reverse ? (args.nseg - 1 - ip) : ip;
+    const int p = seg_of(ip);
     const size_t off = ((size_t)bh * args.nseg + p) * DE;
     const bool more = (ip + 1 < args.nseg);
-    float loc[4];
+    float nxt[4] = {0.f, 0.f, 0.f, 0.f};
+    if (ip + 2 < args.nseg) {
+      const size_t offn = ((size_t)bh * args.nseg + seg_of(ip + 1)) * DE;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) loc[k] = more ? args.buf[off + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] : 0.f;
+      for (int k = 0; k < 4; ++k) nxt[k] = args.buf[offn + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx];
+    }
 #pragma unroll
     for (int k = 0; k < 4; ++k) args.buf[off + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] = z[k];
     if (args.buf_t) {
@@ -328,7 +338,10 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs args, const De
     if (more) {
       const float g = gamma[p];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) z[k] = fmaf(g, z[k], loc[k]);
+      for (int k = 0; k < 4; ++k) {
+        z[k] = fmaf(g, z[k], loc[k]);
+        loc[k] = nxt[k];
+      }
     }
   }
 }

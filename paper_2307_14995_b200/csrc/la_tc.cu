@@ -144,12 +144,14 @@ __device__ __forceinline__ void store_pairs16(__nv_bfloat16* tile, int row, int 
   *reinterpret_cast<uint4*>(tile + row * 64 + (((c8 + 1) ^ (row & 7)) << 3)) = make_uint4(v[4], v[5], v[6], v[7]);
 }
 
-// Optional pipeline trace (debug builds only): thread block 0 stores clock64() at named events.
+// Optional pipeline trace (debug builds with -DLA_TC_TRACE only): one chosen thread block stores
+// clock64() at named events, and every block of a walk launch its start/end time.
 #ifdef LA_TC_TRACE
 __device__ long long* g_tc_trace = nullptr;
+__device__ unsigned int g_tc_trace_block = 0;
 #define TC_TRACE(it, ev)                                                                          \
   do {                                                                                            \
-    if (g_tc_trace && blockIdx.x == 270 && (it) < 64) g_tc_trace[(it) * 32 + (ev)] = clock64();     \
+    if (g_tc_trace && blockIdx.x == g_tc_trace_block && (it) < 64) g_tc_trace[(it) * 32 + (ev)] = clock64();     \
   } while (0)
 __device__ unsigned long long* g_tc_cta_times = nullptr;  // [grid][2] start/end in ns (walk kernels only)
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
@@ -770,8 +772,9 @@ cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int pre
 }
 
 #ifdef LA_TC_TRACE
-extern "C" void la_debug_set_trace(long long* device_buffer) {
+extern "C" void la_debug_set_trace(long long* device_buffer, unsigned int block) {
   cudaMemcpyToSymbol(g_tc_trace, &device_buffer, sizeof(device_buffer));
+  cudaMemcpyToSymbol(g_tc_trace_block, &block, sizeof(block));
 }
 extern "C" void la_debug_set_cta_times(unsigned long long* device_buffer) {
   cudaMemcpyToSymbol(g_tc_cta_times, &device_buffer, sizeof(device_buffer));
