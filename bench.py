@@ -55,6 +55,13 @@ def bytes_per_token_head(d: int, out_bytes: int, what: str) -> float:
     return float({"fwd": fwd, "bwd": bwd, "step": fwd + bwd, "walk": walk}[what])
 
 
+# DRAM traffic of one walk launch per token-head, from the ncu capture summarised in
+# profiles/tc_walk_kernel_small_case.md: (105.46 MB read + 33.91 MB written) / 131072 token-heads.
+# (Reads equal the algorithmic 768 B; about half of the 512 B of output was still in L2 when that
+# small launch ended, so the full-size launch writes more than this figure suggests.)
+WALK_DRAM_BYTES_PER_TOKEN_HEAD = (105.46e6 + 33.91e6) / 131072
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -354,7 +361,9 @@ def run_ours(args):
             "roofline": {"kernel": "block walk (one launch each for O, dQ, dV, dK)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
-                         "traffic": None, "peak_source": peaks["source"],
+                         "traffic": WALK_DRAM_BYTES_PER_TOKEN_HEAD * th,
+                         "traffic_note": "ncu dram bytes of a 131072-token-head launch scaled by token-heads",
+                         "peak_source": peaks["source"],
                          "avg_launch_ms": walk_avg_ms, "launches": walk_n, "bytes_per_launch": walk_bytes},
             "step_roofline": {"t_roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_step,
                               "bytes": step_bytes, "flops": th * F, "peak_source": peaks["source"]},
