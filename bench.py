@@ -193,7 +193,7 @@ def run_reference(args):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2307_14995_b200 import binding as la, inputs
+    from paper_2307_14995_b200 import binding as la, dist_utils, inputs
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -213,11 +213,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return dist_utils.max_over_ranks(x, device=dev)
 
     w = inputs.WORKLOADS[WORKLOAD]
     out_dtype = torch.float32
