@@ -225,7 +225,7 @@ def run_ours(args):
         w = dataclasses.replace(w, H=8, N=16384)
         q, k, v, do = (x[:, :8, :16384].contiguous() for x in (q, k, v, do))
         lam = lam[:8].contiguous()
-    shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype)
+    shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype, precision=args.precision)
     o = torch.empty((w.B, w.H, w.N, w.e), dtype=out_dtype, device=dev)
     dq, dk, dv = (torch.empty((w.B, w.H, w.N, w.d), dtype=out_dtype, device=dev) for _ in range(3))
     ws_f = la.alloc_workspace(la.LA_OP_FWD, shape, dev)
@@ -386,6 +386,9 @@ def main():
     ap.add_argument("--small", action="store_true",
                     help="profiling aid: 8 heads x 16384 tokens of the workload for the fwd+bwd leg")
     ap.add_argument("--decode-steps", type=int, default=0, help="profiling aid: recurrent steps per pass")
+    ap.add_argument("--precision", type=int, default=-1,
+                    help="experiment: LA_SPLIT_* bits for the tensor-core kernels (-1 = library default, all on; "
+                         "anything else does not meet the parity tolerance on every head)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
