@@ -6,17 +6,19 @@
 // tensor cores (tcgen05.mma, fp32 accumulators in tensor memory):
 //   M1  S        = a b^T                          128x128, K = 128
 //   M2  O_inter  = a Z_hi (+ a Z_lo)              128x64,  K = 128   (state of the previous block)
-//   M3  dZ       = b^T [fc_hi | fc_lo]            128x128, K = 128   (fc = diag(f_state) c; halves summed later)
+//   M3  dZ       = b^T fc_hi (+ b^T fc_lo)        128x64,  K = 128   (fc = diag(f_state) c; the state-only
+//                                                                      pre-pass uses one N = 128 product)
 //   M4  O_intra  = P_hi c (+ P_lo c)              128x64,  K = 128   (P = S (.) D, read from tensor memory)
 // and combines out = O_intra + diag(f_out) O_inter, Z <- Gamma Z + dZ on the CUDA
 // cores.  Operands that are formed on chip from fp32 values (P, fc, Z) are carried
 // as two bf16 terms hi + lo = x (to 2^-17), so that the only rounding left is the
 // fp32 accumulation the method prescribes; each split can be turned off.
 //
-// Measured on B200: one tcgen05.mma of M = 128, K = 16 occupies the tensor pipe for
-// about 64 clocks whether N is 64 or 128 (and 128 clocks for N = 256), so the hi and
-// lo halves of M3 share one N = 128 instruction; M2 and M4 stay at N = 64 because
-// tensor memory (512 columns) is full: 2 x 128 (S/P, double-buffered) + 64 + 64 + 128.
+// Tensor memory (512 columns) is full: 2 x 128 (S/P, double-buffered) + 64 (O_intra) +
+// 2 x 64 (O_inter, double-buffered so that M2 of the next block need not wait until the
+// output group has read this block's accumulators) + 64 (dZ).  (Measured on B200: one
+// tcgen05.mma of M = 128, K = 16 occupies the tensor pipe for about 64 clocks whether N is
+// 64 or 128, so the N = 64 products run at half the pipe's rate; wider tiles do not fit.)
 //
 // Warp roles (24 warps; every group has whole multiples of four warps because a warp
 // can only touch the 32-lane quarter of tensor memory given by its index mod 4):
@@ -57,8 +59,8 @@ using namespace ptx;
 
 constexpr int TC_THREADS = 768;
 constexpr int TMEM_COLS = 512;
-// tensor-memory columns: two S/P buffers, O_intra, O_inter, dZ (hi-part | lo-part)
-constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_OI = 256, COL_OE = 320, COL_DZ = 384;
+// tensor-memory columns: two S/P buffers, O_intra, two O_inter buffers, dZ
+constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_OI = 256, COL_OE0 = 320, COL_OE1 = 384, COL_DZ = 448;
 constexpr long long WAIT_BUDGET = 2000000000LL;  // clocks (~1 s)
 
 enum Bar {
@@ -138,10 +140,27 @@ __device__ __forceinline__ void split16(const float (&x)[16], uint32_t (&hi)[8],
   }
 }
 
-// Stores 16 consecutive elements (two 16-byte chunks, chunk index c8 and c8+1) of swizzled row `row`.
-__device__ __forceinline__ void store_pairs16(__nv_bfloat16* tile, int row, int c8, const uint32_t (&v)[8]) {
-  *reinterpret_cast<uint4*>(tile + row * 64 + ((c8 ^ (row & 7)) << 3)) = make_uint4(v[0], v[1], v[2], v[3]);
-  *reinterpret_cast<uint4*>(tile + row * 64 + (((c8 + 1) ^ (row & 7)) << 3)) = make_uint4(v[4], v[5], v[6], v[7]);
+// Eight-element variant (fewer live registers; used where a thread also carries state rows).
+__device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& lo) {
+  __nv_bfloat162 h[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+  float r[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 hf = __bfloat1622float2(h[i]);
+    r[2 * i] = x[2 * i] - hf.x;
+    r[2 * i + 1] = x[2 * i + 1] - hf.y;
+  }
+  uint32_t hw[4], lw[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 l = __floats2bfloat162_rn(r[2 * i], r[2 * i + 1]);
+    hw[i] = *reinterpret_cast<const uint32_t*>(&h[i]);
+    lw[i] = *reinterpret_cast<const uint32_t*>(&l);
+  }
+  hi = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+  lo = make_uint4(lw[0], lw[1], lw[2], lw[3]);
 }
 
 // Optional pipeline trace (debug builds with -DLA_TC_TRACE only): one chosen thread block stores
@@ -266,7 +285,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       constexpr uint32_t ID_MN128 = umma_idesc_bf16(128, 128, true, true); // same with [fc_hi | fc_lo], N = 128
       const uint32_t zh0 = smem_u32(&sm.z_hi[0]), zl0 = smem_u32(&sm.z_lo[0]);
       const uint32_t fh0 = smem_u32(&sm.fc_hi[0]);
-      const uint32_t id_m3 = split_c ? ID_MN128 : ID_MN64;
       if (STATE_ONLY) {
         for (int it = 0; it < nblk; ++it) {
           const int s = it & 1;
@@ -276,10 +294,12 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           TC_WAIT(FULL_B0 + s, par2, 4);
           TC_WAIT(FC_READY0 + s, par2, 5);
           tc_fence_after_sync();
+          // state-only kernel: tensor memory is otherwise unused, so hi and lo share one N = 128
+          // instruction ([fc_hi | fc_lo], 16 KB apart) into columns 0..127; the halves are summed at the end
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            umma_bf16(tmem + COL_DZ, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
-                      umma_desc_sw128(fbuf + k * 2048, 16384, 1024), id_m3, (it > 0 || k > 0));
+            umma_bf16(tmem + COL_S0, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
+                      umma_desc_sw128(fbuf + k * 2048, 16384, 1024), split_c ? ID_MN128 : ID_MN64, (it > 0 || k > 0));
           issued_mma = true;
           umma_commit(&sm.bars[B_FREE0 + s]);
           umma_commit(&sm.bars[FC_FREE0 + s]);
@@ -315,25 +335,32 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 #pragma unroll
           for (int k = 0; k < 8; ++k)
             umma_bf16(tmem + COL_DZ, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
-                      umma_desc_sw128(fh0 + k * 2048, 16384, 1024), id_m3, k > 0);
+                      umma_desc_sw128(fh0 + k * 2048, 16384, 1024), ID_MN64, k > 0);
+          if (split_c) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              umma_bf16(tmem + COL_DZ, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
+                        umma_desc_sw128(fh0 + 16384 + k * 2048, 16384, 1024), ID_MN64, 1);
+          }
           umma_commit(&sm.bars[DZ_READY]);
           umma_commit(&sm.bars[B_FREE0 + s]);
           // M2: O_inter = a Z   (state after the previous block / the entry state)
           TC_WAIT(Z_READY, par1, 12);
-          if (it > 0) TC_WAIT(O_FREE, (it - 1) & 1, 13);
+          // this O_inter buffer was last read for block it-2; that read was already awaited before M4(it-1)
+          const uint32_t col_oe = (it & 1) ? COL_OE1 : COL_OE0;
           tc_fence_after_sync();
           TC_TRACE(it, 5);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
-            umma_bf16(tmem + COL_OE, umma_desc_sw128(a0 + ko, 16, 1024),
+            umma_bf16(tmem + col_oe, umma_desc_sw128(a0 + ko, 16, 1024),
                       umma_desc_sw128(zh0 + k * 2048, 16384, 1024), ID_KN, k > 0);
           }
           if (split_z) {
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
               const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
-              umma_bf16(tmem + COL_OE, umma_desc_sw128(a0 + ko, 16, 1024),
+              umma_bf16(tmem + col_oe, umma_desc_sw128(a0 + ko, 16, 1024),
                         umma_desc_sw128(zl0 + k * 2048, 16384, 1024), ID_KN, 1);
             }
           }
@@ -359,6 +386,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           // M4: O_intra = P c, P read from tensor memory (K step k: hi pairs at column 16k, lo pairs at 16k+8)
           TC_WAIT(P_READY0 + s, par2, 14);
           TC_WAIT(FULL_C0 + s, par2, 15);
+          if (it > 0) TC_WAIT(O_FREE, (it - 1) & 1, 26);  // O_intra of the previous block has been read
           tc_fence_after_sync();
           TC_TRACE(it, 6);
 #pragma unroll
@@ -450,21 +478,20 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     // 4*zh .. 4*zh+3 of the 64-column row), into the swizzled operand buffer at hi_tile / lo_tile.
     auto make_fc = [&](const uint4 (&raw)[4], float f, __nv_bfloat16* hi_tile, __nv_bfloat16* lo_tile) {
 #pragma unroll
-      for (int gg = 0; gg < 2; ++gg) {  // 16 elements per pass
-        const int g = zh * 2 + gg;
-        const uint32_t w[8] = {raw[2 * gg].x, raw[2 * gg].y, raw[2 * gg].z, raw[2 * gg].w,
-                               raw[2 * gg + 1].x, raw[2 * gg + 1].y, raw[2 * gg + 1].z, raw[2 * gg + 1].w};
-        float x16[16];
+      for (int x4 = 0; x4 < 4; ++x4) {  // 8 elements (one 16-byte chunk) per pass: few live registers
+        const uint32_t w[4] = {raw[x4].x, raw[x4].y, raw[x4].z, raw[x4].w};
+        float x8[8];
 #pragma unroll
-        for (int x = 0; x < 8; ++x) {
+        for (int x = 0; x < 4; ++x) {
           const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[x]));
-          x16[2 * x] = v.x * f;
-          x16[2 * x + 1] = v.y * f;
+          x8[2 * x] = v.x * f;
+          x8[2 * x + 1] = v.y * f;
         }
-        uint32_t h8[8], l8[8];
-        split16(x16, h8, l8);
-        store_pairs16(hi_tile, r, 2 * g, h8);
-        if (split_c) store_pairs16(lo_tile, r, 2 * g, l8);
+        uint4 h, l;
+        split8(x8, h, l);
+        const int off = r * 64 + (((4 * zh + x4) ^ (r & 7)) << 3);
+        *reinterpret_cast<uint4*>(hi_tile + off) = h;
+        if (split_c) *reinterpret_cast<uint4*>(lo_tile + off) = l;
       }
       fence_proxy_async_smem();
     };
@@ -509,8 +536,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 #pragma unroll
       for (int pc = 0; pc < 2; ++pc) {
         uint32_t dh[16], dl[16];
-        tmem_ld_x16(lane_addr + COL_DZ + zh * 32 + pc * 16, dh);
-        if (split_c) tmem_ld_x16(lane_addr + COL_DZ + 64 + zh * 32 + pc * 16, dl);
+        tmem_ld_x16(lane_addr + COL_S0 + zh * 32 + pc * 16, dh);
+        if (split_c) tmem_ld_x16(lane_addr + COL_S0 + 64 + zh * 32 + pc * 16, dl);
         tmem_ld_wait();
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -540,14 +567,15 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       // bf16 hi/lo operand of the current state rows (this warp's 32 columns)
       auto write_state_operand = [&]() {
 #pragma unroll
-        for (int gg = 0; gg < 2; ++gg) {
-          float x16[16];
+        for (int x4 = 0; x4 < 4; ++x4) {
+          float x8[8];
 #pragma unroll
-          for (int x = 0; x < 16; ++x) x16[x] = zreg[gg * 16 + x];
-          uint32_t h8[8], l8[8];
-          split16(x16, h8, l8);
-          store_pairs16(sm.z_hi, r, 2 * (zh * 2 + gg), h8);
-          if (split_z) store_pairs16(sm.z_lo, r, 2 * (zh * 2 + gg), l8);
+          for (int x = 0; x < 8; ++x) x8[x] = zreg[x4 * 8 + x];
+          uint4 h, l;
+          split8(x8, h, l);
+          const int off = r * 64 + (((4 * zh + x4) ^ (r & 7)) << 3);
+          *reinterpret_cast<uint4*>(sm.z_hi + off) = h;
+          if (split_z) *reinterpret_cast<uint4*>(sm.z_lo + off) = l;
         }
         fence_proxy_async_smem();
       };
@@ -570,16 +598,11 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           const float gamma = exp2f(-s2 * (float)Cr);
 #pragma unroll
           for (int pc = 0; pc < 2; ++pc) {
-            uint32_t dh[16], dl[16];
+            uint32_t dh[16];
             tmem_ld_x16(lane_addr + COL_DZ + zh * 32 + pc * 16, dh);
-            if (split_c) tmem_ld_x16(lane_addr + COL_DZ + 64 + zh * 32 + pc * 16, dl);
             tmem_ld_wait();
 #pragma unroll
-            for (int x = 0; x < 16; ++x) {
-              float dz = __uint_as_float(dh[x]);
-              if (split_c) dz += __uint_as_float(dl[x]);
-              zreg[pc * 16 + x] = fmaf(gamma, zreg[pc * 16 + x], dz);
-            }
+            for (int x = 0; x < 16; ++x) zreg[pc * 16 + x] = fmaf(gamma, zreg[pc * 16 + x], __uint_as_float(dh[x]));
           }
           tc_fence_before_sync();
           mbar_arrive(&sm.bars[DZ_FREE]);
@@ -635,7 +658,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             const int col = (pass * PIECES + pc) * 16;
             uint32_t oi[16], oe[16];
             tmem_ld_x16(lane_addr + COL_OI + col, oi);
-            tmem_ld_x16(lane_addr + COL_OE + col, oe);
+            tmem_ld_x16(lane_addr + ((it & 1) ? COL_OE1 : COL_OE0) + col, oe);
             tmem_ld_wait();
             if (pass == PASSES - 1 && pc == PIECES - 1) {
               tc_fence_before_sync();
