@@ -234,7 +234,7 @@ def run_ours(args):
 
     def step():
         la.la_fwd(shape, q, k, v, lam, o, None, None, ws_f, stream)
-        la.la_bwd(shape, q, k, v, do, lam, dq, dk, dv, None, None, None, ws_b, stream)
+        la.la_bwd(shape, q, k, v, do, lam, dq, dk, dv, None, None, None, ws_b, stream, fwd_workspace=ws_f)
 
     train_steps = 0 if args.only == "decode" else args.steps
     # clocks are sampled from before the warm-up until the last timed leg has finished

@@ -98,8 +98,9 @@ int la_segment_length(const la_shape* shape);
  *   kv_out  [B,H,d,e] fp32 state after the last token (no extra decay), or NULL.
  * With kv_in the result is o_t = kv_t^T q_t where kv_{-1} = kv_in.
  * workspace: device scratch of at least la_workspace_bytes(LA_OP_FWD, shape)
- * bytes, 256-byte aligned; may be NULL when that size is 0.  Its contents are
- * undefined afterwards.  Calls that share a workspace must be stream-ordered.
+ * bytes, 256-byte aligned; may be NULL when that size is 0.  Calls that share a
+ * workspace must be stream-ordered.  Afterwards the workspace holds the state
+ * entering each segment; la_bwd_reuse can take it to skip recomputing those.
  */
 la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void* v,
                  const float* lambda_host, void* o, const float* kv_in, float* kv_out,
@@ -120,6 +121,18 @@ la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void
                  const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
                  const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * la_bwd that reuses the forward pass's segment states.  fwd_workspace is the workspace
+ * a preceding la_fwd used for the SAME shape (incl. seg_len/path), inputs, lambda and
+ * kv_in, untouched since; the dQ part of Algorithm 4 then starts from those states
+ * instead of re-reading K and V in a pre-pass.  NULL, or a shape with a single segment,
+ * makes it identical to la_bwd.  fwd_workspace must not overlap `workspace`.
+ */
+la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, const void* v,
+                       const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
+                       const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
+                       const void* fwd_workspace, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * One recurrent decode step (one iteration of Algorithm 2) for every (b,h):

@@ -24,7 +24,7 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
-           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc")
+           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
 
@@ -65,6 +65,8 @@ def load():
         lib.la_fwd_noalloc.restype = I
         lib.la_bwd.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.la_bwd.restype = I
+        lib.la_bwd_reuse.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.la_bwd_reuse.restype = I
         lib.la_decode_step.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_step.restype = I
         lib.la_host_arena_bytes.argtypes = [sp]
@@ -185,11 +187,18 @@ def la_fwd_noalloc(shape: LaShape, q, k, v, lam, o, kv_in=None, kv_out=None, str
 
 
 def la_bwd(shape: LaShape, q, k, v, do, lam, dq, dk, dv, kv_in=None, grad_kv_out=None, grad_kv_in=None,
-           workspace=None, stream=None):
+           workspace=None, stream=None, fwd_workspace=None):
+    """fwd_workspace: the workspace of the matching la_fwd call (same shape, inputs, kv_in), to reuse its
+    segment states (la_bwd_reuse); None recomputes them (la_bwd)."""
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    rc = load().la_bwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(do), _lam(lam), _ptr(dq),
-                       _ptr(dk), _ptr(dv), _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in),
-                       _ptr(workspace), ws_bytes, _stream(stream))
+    if fwd_workspace is None:
+        rc = load().la_bwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(do), _lam(lam), _ptr(dq),
+                           _ptr(dk), _ptr(dv), _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in),
+                           _ptr(workspace), ws_bytes, _stream(stream))
+    else:
+        rc = load().la_bwd_reuse(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(do), _lam(lam), _ptr(dq),
+                                 _ptr(dk), _ptr(dv), _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in),
+                                 _ptr(fwd_workspace), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_bwd")
 

@@ -264,12 +264,20 @@ la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void
                  const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
                  const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
                  void* workspace, size_t workspace_bytes, void* stream) {
+  return la_bwd_reuse(shape, q, k, v, d_o, lambda_host, dq, dk, dv, kv_in, grad_kv_out, grad_kv_in, nullptr,
+                      workspace, workspace_bytes, stream);
+}
+
+la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, const void* v,
+                       const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
+                       const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
+                       const void* fwd_workspace, void* workspace, size_t workspace_bytes, void* stream) {
   la_status st = check_shape(shape, true);
   if (st != LA_OK) return st;
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return LA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv) || !aligned16(kv_in) || !aligned16(grad_kv_out) ||
-      !aligned16(grad_kv_in))
+      !aligned16(grad_kv_in) || !aligned16(fwd_workspace))
     return LA_ERR_INVALID_ARG;
   DecayTable tab;
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
@@ -277,6 +285,7 @@ la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void
   if ((st = make_plan(shape, &p)) != LA_OK) return st;
   const size_t one = state_set_bytes(shape, p);
   if (!workspace || workspace_bytes < 3 * one) return LA_ERR_WORKSPACE;
+  if (fwd_workspace == workspace) return LA_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LA_ERR_INVALID_ARG;
   if ((st = check_device()) != LA_OK) return st;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
@@ -288,8 +297,13 @@ la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void
 
   // dQ = fwd(a = dO, b = V, c = K); its state is KV^T, so the caller's kv_in enters transposed.
   const float* entry_q = nullptr;
-  if (multi) LA_TRY_CUDA(run_prepass(shape, p, tab, v, k, 0, buf_kvt, cs));
-  if (multi || kv_in) {
+  if (multi && fwd_workspace) {
+    // la_fwd left KV entering each segment (kv_in included) in its workspace: transpose, no pre-pass
+    LA_TRY_CUDA(launch_transpose_states(static_cast<const float*>(fwd_workspace), buf_kvt, (long)p.BH * p.nseg,
+                                        shape->d, shape->e, cs));
+    entry_q = buf_kvt;
+  } else if (multi || kv_in) {
+    if (multi) LA_TRY_CUDA(run_prepass(shape, p, tab, v, k, 0, buf_kvt, cs));
     LA_TRY_CUDA(run_scan(shape, p, tab, buf_kvt, nullptr, kv_in, true, 0, cs));
     entry_q = buf_kvt;
   }
@@ -337,7 +351,7 @@ size_t la_host_arena_bytes(const la_shape* shape) {
   size_t total = 0;
   total += 2 * round256(tokens * shape->d * in_sz) + 2 * round256(tokens * shape->e * in_sz);
   total += 2 * round256(tokens * shape->d * out_sz) + 2 * round256(tokens * shape->e * out_sz);
-  total += round256(wf > wb ? wf : wb);
+  total += round256(wf) + round256(wb);
   return total;
 }
 
@@ -369,8 +383,10 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
   LA_TRY_CUDA(cudaMemcpyAsync(ddo_in, d_o_host, bv, cudaMemcpyHostToDevice, cs));
   la_status st = la_fwd(shape, dq_in, dk_in, dv_in, lambda_host, d_o, nullptr, nullptr, ws, ws_bytes, stream);
   if (st != LA_OK) return st;
-  st = la_bwd(shape, dq_in, dk_in, dv_in, ddo_in, lambda_host, d_dq, d_dk, d_dv, nullptr, nullptr,
-              nullptr, ws, ws_bytes, stream);
+  // the forward workspace (first state set) feeds the backward pass, which uses the space behind it
+  const size_t wf = round256(la_workspace_bytes(LA_OP_FWD, shape));
+  st = la_bwd_reuse(shape, dq_in, dk_in, dv_in, ddo_in, lambda_host, d_dq, d_dk, d_dv, nullptr, nullptr, nullptr,
+                    wf > 0 ? ws : nullptr, ws + wf, ws_bytes - wf, stream);
   if (st != LA_OK) return st;
   LA_TRY_CUDA(cudaMemcpyAsync(o_host, d_o, bdv, cudaMemcpyDeviceToHost, cs));
   LA_TRY_CUDA(cudaMemcpyAsync(dq_host, d_dq, bdq, cudaMemcpyDeviceToHost, cs));

@@ -67,6 +67,8 @@ cudaError_t launch_simt_walk(const OpArgs& args, const DecayTable& tab, int Da, 
 cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int Da, int Ec, int in_dt,
                                 cudaStream_t stream);
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream);
+// dst[m] = transpose(src[m]) for `count` row-major Da x Ec fp32 matrices.
+cudaError_t launch_transpose_states(const float* src, float* dst, long count, int Da, int Ec, cudaStream_t stream);
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv, void* o, int BH,
                           int H, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
                           cudaStream_t stream);

@@ -421,6 +421,32 @@ cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int D
   return cudaErrorInvalidValue;
 }
 
+// dst[m] = src[m]^T for `count` row-major Da x Ec matrices (32x32 tiles through shared memory).
+__global__ void __launch_bounds__(256) transpose_states_kernel(const float* __restrict__ src, float* __restrict__ dst,
+                                                               int Da, int Ec) {
+  __shared__ float tile[32][33];
+  const size_t m = blockIdx.x;
+  const int tiles_y = Ec / 32;
+  const int x0 = (blockIdx.y / tiles_y) * 32, y0 = (blockIdx.y % tiles_y) * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const float* s = src + m * Da * Ec;
+  float* d = dst + m * Da * Ec;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) tile[ty + 8 * k][tx] = s[(size_t)(x0 + ty + 8 * k) * Ec + y0 + tx];
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < 4; ++k) d[(size_t)(y0 + ty + 8 * k) * Da + x0 + tx] = tile[tx][ty + 8 * k];
+}
+
+cudaError_t launch_transpose_states(const float* src, float* dst, long count, int Da, int Ec, cudaStream_t stream) {
+  if ((Da % 32) != 0 || (Ec % 32) != 0 || count < 1 || count > 2147483647L) return cudaErrorInvalidValue;
+  const dim3 grid((unsigned)count, (unsigned)((Da / 32) * (Ec / 32)));
+  KernelTimer timer(K_SCAN, stream);
+  transpose_states_kernel<<<grid, 256, 0, stream>>>(src, dst, Da, Ec);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream) {
   if (args.nseg > SCAN_MAX_SEG || (args.Da % 32) != 0 || (args.Ec % 32) != 0) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)args.BH, (unsigned)((args.Da / 32) * (args.Ec / 32)));

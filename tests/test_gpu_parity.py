@@ -389,3 +389,31 @@ def test_errors_on_device():
         la.fwd(qg, kg, vg, torch.tensor([1.0, 0.0]))
     with pytest.raises(la.LaError):
         la.fwd(qg, kg, vg, torch.tensor([1.0, 2.0]))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_backward_reusing_forward_segment_states(path):
+    """la_bwd_reuse: the dQ walk starts from the states la_fwd left in its workspace (no pre-pass)."""
+    d = 128
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N, seg_len = 2, 3, 1100, 256
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=17)
+    lam = torch.tensor([1.0, 0.98, 0.5])
+    kv_in = inputs.make_state(B, H, d, d, seed=18)
+    gko = inputs.make_state(B, H, d, d, seed=19)
+    qg, kg, vg, dog, kin, gk = to_dev(q, k, v, do, kv_in, gko)
+    shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, seg_len, path)
+    o = torch.empty((B, H, N, d), dtype=torch.float32, device=DEV)
+    dq, dk, dv = (torch.empty((B, H, N, d), dtype=torch.float32, device=DEV) for _ in range(3))
+    gin = torch.empty((B, H, d, d), dtype=torch.float32, device=DEV)
+    ws_f = la.alloc_workspace(la.LA_OP_FWD, shape, DEV)
+    ws_b = la.alloc_workspace(la.LA_OP_BWD, shape, DEV)
+    la.la_fwd(shape, qg, kg, vg, lam, o, kin, None, ws_f)
+    la.la_bwd(shape, qg, kg, vg, dog, lam, dq, dk, dv, kin, gk, gin, ws_b, fwd_workspace=ws_f)
+    torch.cuda.synchronize()
+    la.device_status()
+    ref = oracle_all(q, k, v, do, lam, kv_in.double().numpy(), gko.double().numpy())
+    tol = TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4
+    for n, g, r in zip(("o", "dq", "dk", "dv", "grad_kv_in"), (o, dq, dk, dv, gin), (ref[0], ref[2], ref[3], ref[4], ref[5])):
+        assert_close(g, r, tol, n)
