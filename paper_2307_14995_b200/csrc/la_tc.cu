@@ -68,7 +68,7 @@ enum Bar {
   A_FREE0, A_FREE1, B_FREE0, B_FREE1, C_FREE0, C_FREE1,       // consumers -> TMA
   S_READY0, S_READY1, P_READY0, P_READY1,
   FC_READY0, FC_READY1, FC_FREE0, FC_FREE1,                   // (second buffer: state-only kernel)
-  DZ_READY, DZ_FREE, Z_READY, Z_FREE, O_READY, O_FREE, DRAIN,
+  DZ_READY, DZ_FREE, Z_READY, Z_FREE, O_READY, O_FREE, OG_SYNC, DRAIN,
   NUM_BARS
 };
 
@@ -84,7 +84,6 @@ struct alignas(1024) TcSmem {
   __nv_bfloat16 fc_lo[128 * 64];
   __nv_bfloat16 z_hi[128 * 64];   // state operand; in the state-only kernel: second fc buffer
   __nv_bfloat16 z_lo[128 * 64];
-  float dtab[128];
   uint64_t bars[NUM_BARS];
   uint32_t tmem_slot;
   int abort;
@@ -196,10 +195,32 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     }                                                                    \
   } while (0)
 
+// The same for a whole warp waiting together: the outcome is made warp-uniform so that the
+// warp-level synchronisation of the elected arrivals below can never be entered by a part of a warp.
+#define TC_WAIT_WARP(barid, par, code)                                                    \
+  do {                                                                                    \
+    const bool ok_ = wait_or_abort(&sm.bars[barid], (par), &sm.abort);                    \
+    if (!__all_sync(0xffffffffu, ok_)) {                                                  \
+      if (!ok_ && !sm.abort) atomicCAS(&g_tc_status, 0u, (unsigned)(code));               \
+      sm.abort = 1;                                                                       \
+      goto teardown;                                                                      \
+    }                                                                                     \
+  } while (0)
+
+// One arrival per warp: every lane has fenced its own writes, the warp synchronises, lane 0
+// arrives.  (A barrier that 256 threads arrive on costs 256 serialised shared-memory atomics per
+// phase; at six such barriers per block that was a third of the kernel's shared-memory traffic.)
+#define WARP_ARRIVE(barid)                               \
+  do {                                                   \
+    __syncwarp();                                        \
+    if (lane == 0) mbar_arrive(&sm.bars[barid]);         \
+  } while (0)
+
 template <bool REV, bool STATE_ONLY, typename TOut>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-          const __grid_constant__ CUtensorMap tm_c, const TcArgs args, const DecayTable tab) {
+          const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_out, const TcArgs args,
+          const DecayTable tab) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler keeps
   // the shared address space (ld.shared / st.shared rather than generic accesses)
@@ -221,10 +242,12 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   if (tid == 0) {
     for (int i = 0; i < NUM_BARS; ++i) {
       uint32_t count = 1;
+      // barriers that a compute group arrives on: one arrival per warp
       if (i == P_READY0 || i == P_READY1 || i == FC_READY0 || i == FC_READY1 || i == Z_READY || i == DZ_FREE)
-        count = 256;
-      if (i == O_FREE) count = 128;
-      if (i == C_FREE0 || i == C_FREE1) count = STATE_ONLY ? 256 : 128;  // the threads that last touch the c tile
+        count = 8;
+      if (i == O_FREE || i == OG_SYNC) count = 4;
+      // the c tile is released by the warps that read it (state-only) / by the thread that stores from it (walk)
+      if (i == C_FREE0 || i == C_FREE1) count = STATE_ONLY ? 8 : 1;
       mbar_init(&sm.bars[i], count);
     }
     sm.abort = 0;
@@ -232,12 +255,12 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     tma_prefetch_desc(&tm_a);
     tma_prefetch_desc(&tm_b);
     tma_prefetch_desc(&tm_c);
+    if (!STATE_ONLY) tma_prefetch_desc(&tm_out);
   }
   if (warp == 1) {
     tmem_alloc(&sm.tmem_slot, TMEM_COLS);
     tmem_relinquish();
   }
-  if (tid < 128) sm.dtab[tid] = exp2f(-s2 * (float)tid);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -413,7 +436,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       for (int it = 0; it < nblk; ++it) {
         const int s = it & 1;
         const uint32_t colS = lane_addr + (s ? COL_S1 : COL_S0);
-        TC_WAIT(S_READY0 + s, (it >> 1) & 1, 17);
+        TC_WAIT_WARP(S_READY0 + s, (it >> 1) & 1, 17);
         tc_fence_after_sync();
         if (tid == 224) TC_TRACE(it, 7);
 #pragma unroll 1
@@ -430,12 +453,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
               uint32_t sreg[16];
               tmem_ld_x16(colS + cc * 32 + hh * 16, sreg);
               float d[16];
+              // lambda^n on the special-function unit (idle otherwise); n < 0 is masked out below
+              const float n0 = (float)(REV ? (cc * 32 + hh * 16 - r) : (r - cc * 32 - hh * 16));
 #pragma unroll
-              for (int x = 0; x < 16; ++x) {
-                const int j = cc * 32 + hh * 16 + x;
-                const int n = REV ? (j - r) : (r - j);
-                d[x] = sm.dtab[n & 127];
-              }
+              for (int x = 0; x < 16; ++x) d[x] = ex2_approx(-s2 * (REV ? n0 + (float)x : n0 - (float)x));
               tmem_ld_wait();
 #pragma unroll
               for (int x = 0; x < 16; ++x) {
@@ -453,7 +474,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
         tmem_st_wait();
         tc_fence_before_sync();
-        mbar_arrive(&sm.bars[P_READY0 + s]);
+        WARP_ARRIVE(P_READY0 + s);
         if (tid == 224) TC_TRACE(it, 8);
       }
     }
@@ -521,16 +542,16 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     if (STATE_ONLY) {
       for (int it = 0; it < nblk; ++it) {
         const int s = it & 1;
-        TC_WAIT(FULL_C0 + s, (it >> 1) & 1, 18);
-        if (it >= 2) TC_WAIT(FC_FREE0 + s, ((it >> 1) - 1) & 1, 19);  // the MMA two blocks back has read this buffer
+        TC_WAIT_WARP(FULL_C0 + s, (it >> 1) & 1, 18);
+        if (it >= 2) TC_WAIT_WARP(FC_FREE0 + s, ((it >> 1) - 1) & 1, 19);  // the MMA two blocks back has read this buffer
         uint4 craw[4];
         c_from_tile(it, craw);
         make_fc(craw, state_factor(it), s ? sm.z_hi : sm.fc_hi, s ? sm.z_lo : sm.fc_lo);
-        mbar_arrive(&sm.bars[FC_READY0 + s]);
-        mbar_arrive(&sm.bars[C_FREE0 + s]);
+        WARP_ARRIVE(FC_READY0 + s);
+        if (lane == 0) mbar_arrive(&sm.bars[C_FREE0 + s]);
       }
       // segment-local state = accumulated dZ (hi-part + lo-part)
-      TC_WAIT(DZ_READY, 0, 20);
+      TC_WAIT_WARP(DZ_READY, 0, 20);
       tc_fence_after_sync();
       float* dst = args.local_out + ((size_t)bh * args.nseg + seg) * (128 * 128) + (size_t)r * 128 + ehalf * 64 + zh * 32;
 #pragma unroll
@@ -580,18 +601,18 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         fence_proxy_async_smem();
       };
       write_state_operand();
-      mbar_arrive(&sm.bars[Z_READY]);
+      WARP_ARRIVE(Z_READY);
       uint4 cnext[4];  // row slice of the next block's c, fetched one block ahead
       c_from_global(0, cnext);
       make_fc(cnext, state_factor(0), sm.fc_hi, sm.fc_lo);
-      mbar_arrive(&sm.bars[FC_READY0]);
+      WARP_ARRIVE(FC_READY0);
       if (nblk > 1) c_from_global(1, cnext);
 
       for (int it = 0; it < nblk; ++it) {
         const int blk = REV ? (nblk - 1 - it) : it;
         const int Cr = min(128, seg_t1 - (seg_t0 + blk * 128));
         // ---- Z <- Gamma Z + dZ ----
-        TC_WAIT(DZ_READY, it & 1, 22);
+        TC_WAIT_WARP(DZ_READY, it & 1, 22);
         tc_fence_after_sync();
         if (tid == 384) TC_TRACE(it, 9);
         {
@@ -605,18 +626,18 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             for (int x = 0; x < 16; ++x) zreg[pc * 16 + x] = fmaf(gamma, zreg[pc * 16 + x], __uint_as_float(dh[x]));
           }
           tc_fence_before_sync();
-          mbar_arrive(&sm.bars[DZ_FREE]);
+          WARP_ARRIVE(DZ_FREE);
         }
         if (it + 1 < nblk) {
           // DZ_READY also says M3 of this block is done, so the fc buffer may be rewritten
           make_fc(cnext, state_factor(it + 1), sm.fc_hi, sm.fc_lo);
-          mbar_arrive(&sm.bars[FC_READY0]);
+          WARP_ARRIVE(FC_READY0);
           if (it + 2 < nblk) c_from_global(it + 2, cnext);
           if (tid == 384) TC_TRACE(it, 10);
           // Z_FREE: M2 of this block has read the old state operand
-          TC_WAIT(Z_FREE, it & 1, 23);
+          TC_WAIT_WARP(Z_FREE, it & 1, 23);
           write_state_operand();
-          mbar_arrive(&sm.bars[Z_READY]);
+          WARP_ARRIVE(Z_READY);
           if (tid == 384) TC_TRACE(it, 11);
         }
       }
@@ -634,6 +655,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       const int q = warp & 3;
       const int r = q * 32 + lane;  // output row i
       const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+      uint32_t og_uses = 0;  // phases of the group's own barrier used so far
       for (int it = 0; it < nblk; ++it) {
         const int s = it & 1;
         const int blk = REV ? (nblk - 1 - it) : it;
@@ -641,11 +663,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         const int Cr = min(128, seg_t1 - t0);
         float f = 0.f;
         if (r < Cr) f = REV ? exp2f(-s2 * (float)(Cr - 1 - r)) : exp2f(-s2 * (float)(r + 1));
-        // 4 KB per warp inside the c tile of this block, which is dead once M4 is done
-        unsigned char* scratch = reinterpret_cast<unsigned char*>(&sm.st[s].c[0]) + q * 4096;
-        TOut* obase = static_cast<TOut*>(args.out) + ((size_t)bh * args.N + t0 + q * 32) * 128 + ehalf * 64;
+        // staging tile for the bulk stores: the c tile of this block, dead once M4 is done
+        unsigned char* stg = reinterpret_cast<unsigned char*>(&sm.st[s].c[0]);
         // O_READY: every MMA up to M4 of this block is done
-        TC_WAIT(O_READY, it & 1, 25);
+        TC_WAIT_WARP(O_READY, it & 1, 25);
         tc_fence_after_sync();
         if (tid == 736) TC_TRACE(it, 12);
         constexpr int PASSES = (sizeof(TOut) == 4) ? 2 : 1;  // 128 bytes of each output row per pass
@@ -662,7 +683,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             tmem_ld_wait();
             if (pass == PASSES - 1 && pc == PIECES - 1) {
               tc_fence_before_sync();
-              mbar_arrive(&sm.bars[O_FREE]);  // both accumulators are in registers now
+              WARP_ARRIVE(O_FREE);  // both accumulators are in registers now
               if (tid == 736) TC_TRACE(it, 13);
             }
             if (sizeof(TOut) == 4) {
@@ -679,30 +700,40 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
               }
             }
           }
+          if (pass > 0) {
+            // the staging tile still feeds the previous pass's store until its source has been read
+            if (warp == 20 && lane == 0) tma_store_wait_read();
+            WARP_ARRIVE(OG_SYNC);
+            TC_WAIT_WARP(OG_SYNC, og_uses & 1, 27);
+            ++og_uses;
+          }
+          // row r of the [128 rows][128 bytes] staging tile, 16-byte chunks swizzled as the store expects
 #pragma unroll
           for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(scratch + lane * 128 + ((c ^ (lane & 7)) << 4)) =
+            *reinterpret_cast<uint4*>(stg + r * 128 + ((c ^ (r & 7)) << 4)) =
                 make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-          __syncwarp();
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const int rowl = 4 * k + (lane >> 3), chunk = lane & 7;
-            const uint4 v = *reinterpret_cast<const uint4*>(scratch + rowl * 128 + ((chunk ^ (rowl & 7)) << 4));
-            if (q * 32 + rowl < Cr) {
-              unsigned char* dst = reinterpret_cast<unsigned char*>(obase + (size_t)rowl * 128) + pass * 128 + chunk * 16;
-              *reinterpret_cast<uint4*>(dst) = v;
-            }
+          fence_proxy_async_smem();
+          WARP_ARRIVE(OG_SYNC);
+          TC_WAIT_WARP(OG_SYNC, og_uses & 1, 28);
+          ++og_uses;
+          if (warp == 20 && lane == 0) {
+            // rows beyond N are clipped by the tensor map (a ragged block is always the last of the sequence)
+            tma_store_3d(&tm_out, stg, ehalf * 64 + pass * (int)(128 / sizeof(TOut)), t0, bh);
+            tma_store_commit();
           }
-          __syncwarp();
         }
-        fence_proxy_async_smem();
-        mbar_arrive(&sm.bars[C_FREE0 + s]);
+        if (warp == 20 && lane == 0) {
+          tma_store_wait_read();
+          mbar_arrive(&sm.bars[C_FREE0 + s]);  // the c tile of this stage may be reloaded
+        }
         if (tid == 736) TC_TRACE(it, 14);
       }
     }
   }
 
 teardown:
+  // the storing thread's bulk stores must have read their shared-memory source before the block exits
+  if (!STATE_ONLY && warp == 20 && lane == 0) tma_store_wait_all();
   // After an expired wait: drain what this thread started so nothing is in flight when the
   // block exits (loads into shared memory, tensor-core work on tensor memory).
   if (sm.abort) {
@@ -740,29 +771,30 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over a bf16 [BH, N, 128] tensor (feature dimension innermost) with a box of
-// 64 x 128 rows x 1 and 128-byte swizzle; rows beyond N read as zero.
-bool make_map(CUtensorMap* m, const void* ptr, int N, int BH) {
+// Tensor map over a [BH, N, 128] tensor (feature dimension innermost) of bf16 or fp32 with a box of
+// 128 bytes x 128 rows x 1 and 128-byte swizzle; rows beyond N read as zero and are not written.
+bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, bool f32 = false) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
+  const cuuint64_t esz = f32 ? 4 : 2;
   cuuint64_t dims[3] = {128, (cuuint64_t)N, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {128 * 2, (cuuint64_t)N * 128 * 2};
-  cuuint32_t box[3] = {64, 128, 1};
+  cuuint64_t strides[2] = {128 * esz, (cuuint64_t)N * 128 * esz};
+  cuuint32_t box[3] = {(cuuint32_t)(128 / esz), 128, 1};
   cuuint32_t es[3] = {1, 1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr),
+             dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <bool REV, bool STATE_ONLY, typename TOut>
-cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
+cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mo,
                      const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
   const size_t smem = sizeof(TcSmem) + 1024;
   auto kern = tc_kernel<REV, STATE_ONLY, TOut>;
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   KernelTimer timer(STATE_ONLY ? K_PREPASS : K_WALK, stream);
-  kern<<<(unsigned)(ta.BH * ta.nseg * 2), TC_THREADS, smem, stream>>>(ma, mb, mc, ta, tab);
+  kern<<<(unsigned)(ta.BH * ta.nseg * 2), TC_THREADS, smem, stream>>>(ma, mb, mc, mo, ta, tab);
   count_launch();
   return cudaGetLastError();
 }
@@ -773,17 +805,17 @@ bool tc_supported() { return encode_fn() != nullptr; }
 
 cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int out_dt, int precision,
                            cudaStream_t stream) {
-  CUtensorMap ma, mb, mc;
+  CUtensorMap ma, mb, mc, mo;
   const bool f32 = (out_dt == DT_F32);
   if (!make_map(&ma, args.a, args.N, args.BH) || !make_map(&mb, args.b, args.N, args.BH) ||
-      !make_map(&mc, args.c, args.N, args.BH))
+      !make_map(&mc, args.c, args.N, args.BH) || !make_map(&mo, args.out, args.N, args.BH, f32))
     return cudaErrorInvalidValue;
   TcArgs ta{args.c, args.out, args.entry, nullptr, args.final_out, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
   if (args.reverse)
-    return f32 ? launch_t<true, false, float>(ma, mb, mc, ta, tab, stream)
-               : launch_t<true, false, __nv_bfloat16>(ma, mb, mc, ta, tab, stream);
-  return f32 ? launch_t<false, false, float>(ma, mb, mc, ta, tab, stream)
-             : launch_t<false, false, __nv_bfloat16>(ma, mb, mc, ta, tab, stream);
+    return f32 ? launch_t<true, false, float>(ma, mb, mc, mo, ta, tab, stream)
+               : launch_t<true, false, __nv_bfloat16>(ma, mb, mc, mo, ta, tab, stream);
+  return f32 ? launch_t<false, false, float>(ma, mb, mc, mo, ta, tab, stream)
+             : launch_t<false, false, __nv_bfloat16>(ma, mb, mc, mo, ta, tab, stream);
 }
 
 cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int precision, cudaStream_t stream) {
@@ -791,9 +823,9 @@ cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int pre
   if (!make_map(&mb, args.b, args.N, args.BH) || !make_map(&mc, args.c, args.N, args.BH))
     return cudaErrorInvalidValue;
   TcArgs ta{args.c, nullptr, nullptr, args.local_out, nullptr, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
-  // the a map is unused by the state-only kernel; pass a valid descriptor anyway
-  return args.reverse ? launch_t<true, true, float>(mb, mb, mc, ta, tab, stream)
-                      : launch_t<false, true, float>(mb, mb, mc, ta, tab, stream);
+  // the a and out maps are unused by the state-only kernel; pass valid descriptors anyway
+  return args.reverse ? launch_t<true, true, float>(mb, mb, mc, mc, ta, tab, stream)
+                      : launch_t<false, true, float>(mb, mb, mc, mc, ta, tab, stream);
 }
 
 #ifdef LA_TC_TRACE
