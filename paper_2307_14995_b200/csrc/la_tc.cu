@@ -167,9 +167,9 @@ __device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& lo
 #ifdef LA_TC_TRACE
 __device__ long long* g_tc_trace = nullptr;
 __device__ unsigned int g_tc_trace_block = 0;
-#define TC_TRACE(it, ev)                                                                          \
-  do {                                                                                            \
-    if (g_tc_trace && blockIdx.x == g_tc_trace_block && (it) < 64) g_tc_trace[(it) * 32 + (ev)] = clock64();     \
+#define TC_TRACE(it, ev)                                                    \
+  do {                                                                      \
+    if (trace_ptr && (it) < 64) trace_ptr[(it) * 32 + (ev)] = clock64();    \
   } while (0)
 __device__ unsigned long long* g_tc_cta_times = nullptr;  // [grid][2] start/end in ns (walk kernels only)
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
@@ -227,6 +227,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef LA_TC_TRACE
+  long long* const trace_ptr = (blockIdx.x == g_tc_trace_block) ? g_tc_trace : nullptr;
+#endif
   const int ehalf = blockIdx.x & 1;
   const int segid = blockIdx.x >> 1;
   const int bh = segid / args.nseg, seg = segid % args.nseg;
@@ -278,6 +281,15 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         const int blk = REV ? (nblk - 1 - it) : it;
         const int t0 = seg_t0 + blk * 128;
         Stage& stg = sm.st[s];
+        // State-only kernel: its two stages hold less than what must be in flight to cover the latency of
+        // HBM, so the tiles two blocks ahead are pulled into L2 now and the loads proper become L2 hits
+        // (measured: 0.276 -> 0.245 ms per launch; the same in the walk kernel made it slower).
+        if (STATE_ONLY && it + 2 < nblk) {
+          const int tp = seg_t0 + (REV ? (nblk - 3 - it) : (it + 2)) * 128;
+          tma_prefetch_3d(&tm_b, 0, tp, bh);
+          tma_prefetch_3d(&tm_b, 64, tp, bh);
+          tma_prefetch_3d(&tm_c, ehalf * 64, tp, bh);
+        }
         if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
         mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], 32768);
         tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
@@ -351,6 +363,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           const uint32_t c0 = smem_u32(&sm.st[s].c[0]);
           const uint32_t col_p = s ? COL_S1 : COL_S0;
           // M3: dZ = b^T [fc_hi | fc_lo]  (needs the previous dZ to have been read)
+          TC_TRACE(it, 15);
           TC_WAIT(FC_READY0, par1, 8);
           if (it > 0) TC_WAIT(DZ_FREE, (it - 1) & 1, 9);
           tc_fence_after_sync();
@@ -367,6 +380,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           }
           umma_commit(&sm.bars[DZ_READY]);
           umma_commit(&sm.bars[B_FREE0 + s]);
+          TC_TRACE(it, 16);
           // M2: O_inter = a Z   (state after the previous block / the entry state)
           TC_WAIT(Z_READY, par1, 12);
           // this O_inter buffer was last read for block it-2; that read was already awaited before M4(it-1)
@@ -389,6 +403,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           }
           umma_commit(&sm.bars[Z_FREE]);
           umma_commit(&sm.bars[A_FREE0 + s]);  // M1 and M2 of this block are done with the a tile
+          TC_TRACE(it, 19);
           // M1 of the next block, into the other S/P buffer
           if (it + 1 < nblk) {
             const int s1 = s ^ 1;
@@ -407,6 +422,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             umma_commit(&sm.bars[S_READY0 + s1]);
           }
           // M4: O_intra = P c, P read from tensor memory (K step k: hi pairs at column 16k, lo pairs at 16k+8)
+          TC_TRACE(it, 20);
           TC_WAIT(P_READY0 + s, par2, 14);
           TC_WAIT(FULL_C0 + s, par2, 15);
           if (it > 0) TC_WAIT(O_FREE, (it - 1) & 1, 26);  // O_intra of the previous block has been read
@@ -423,6 +439,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                            ID_KN, 1);
           }
           umma_commit(&sm.bars[O_READY]);
+          TC_TRACE(it, 21);
         }
       }
     }

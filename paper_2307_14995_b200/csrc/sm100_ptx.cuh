@@ -96,6 +96,12 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
       "r"(c2)
       : "memory");
 }
+// Brings a box into L2 only (no shared-memory destination, no barrier).
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* m, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(reinterpret_cast<uint64_t>(m)),
+               "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, const void* smem_src, int c0, int c1,
                                              int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
@@ -139,6 +145,14 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
   d |= (uint64_t)2 << 61;                              // layout type: 128-byte swizzle
   return d;
 }
+// The same descriptor as two 32-bit halves.  Only the low half depends on the address, and a
+// byte offset `off` (multiple of 16) inside one buffer moves it by off >> 4 (shared-memory
+// addresses stay below 2^18, so the 14-bit field cannot carry).
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+  return ((smem_addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+constexpr uint32_t UMMA_DESC_HI_SBO1024 = (1024u >> 4) | (1u << 14) | (2u << 29);  // sbo = 1024, version, 128-byte swizzle
+
 // Instruction descriptor for kind::f16 with bf16 A/B and fp32 accumulation.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
   return (1u << 4)                       // D format: f32
@@ -212,6 +226,51 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// ---- warp-convergent issue -------------------------------------------------------------------------
+// The MMA-issuing warp runs its whole loop with all 32 lanes converged and only predicates the
+// tcgen05 instructions themselves on one elected lane.  Measured on B200: issued from inside a
+// divergent `if (lane == 0)` region, an MMA costs the issuing warp enough instruction slots that
+// arithmetic-heavy warps on the same scheduler stretch it from 48 to 122 clocks per instruction;
+// issued convergently (operands stay warp-uniform) it stays at the tensor pipe's own 46 clocks.
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t el;
+  asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(el));
+  return el;
+}
+// D[tmem] (+)= A[smem] * B[smem] with descriptors as (low half, common high half); takes effect only
+// in lanes with go != 0.
+__device__ __forceinline__ void umma_bf16_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                             uint32_t idesc, uint32_t accumulate, uint32_t go) {
+  asm volatile(
+      "{\n\t.reg .pred p, g;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 g, %6, 0;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "@g tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(go)
+      : "memory");
+}
+// Same with A in tensor memory.
+__device__ __forceinline__ void umma_bf16_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                                uint32_t idesc, uint32_t accumulate, uint32_t go) {
+  asm volatile(
+      "{\n\t.reg .pred p, g;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 g, %6, 0;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "@g tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(go)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_if(uint64_t* bar, uint32_t go) {
+  asm volatile(
+      "{\n\t.reg .pred g;\n\tsetp.ne.b32 g, %1, 0;\n\t"
+      "@g tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(smem_u32(bar)),
+      "r"(go)
       : "memory");
 }
 
