@@ -247,10 +247,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       uint32_t count = 1;
       // barriers that a compute group arrives on: one arrival per warp
       if (i == P_READY0 || i == P_READY1 || i == FC_READY0 || i == FC_READY1 || i == Z_READY || i == DZ_FREE)
-        count = 8;
+        count = (STATE_ONLY && (i == FC_READY0 || i == FC_READY1)) ? 16 : 8;
       if (i == O_FREE || i == OG_SYNC) count = 4;
       // the c tile is released by the warps that read it (state-only) / by the thread that stores from it (walk)
-      if (i == C_FREE0 || i == C_FREE1) count = STATE_ONLY ? 8 : 1;
+      if (i == C_FREE0 || i == C_FREE1) count = STATE_ONLY ? 16 : 1;
       mbar_init(&sm.bars[i], count);
     }
     sm.abort = 0;
@@ -443,6 +443,71 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
       }
     }
+  } else if (STATE_ONLY && warp >= 4 && warp < 20) {
+    // ------------------------------------ state-only kernel: fc producers ------------------------------------
+    // Sixteen warps (the walk kernel's P and Z groups) form fc = diag(f_state) c: row r = 32 (w % 4) + lane,
+    // sixteen of the 64 value columns each (two 16-byte chunks), hi and lo written to the buffer of stage s.
+    const int w16 = warp - 4, q = w16 & 3, cq = w16 >> 2;
+    const int r = q * 32 + lane;
+    for (int it = 0; it < nblk; ++it) {
+      const int s = it & 1;
+      const int blk = REV ? (nblk - 1 - it) : it;
+      const int t0 = seg_t0 + blk * 128;
+      // decay from token t0 + r to the edge of the segment that the state leaves through
+      float f = 0.f;
+      if (r < min(128, seg_t1 - t0))
+        f = REV ? exp2f(-s2 * (float)(t0 + r - seg_t0 + 1)) : exp2f(-s2 * (float)(seg_t1 - 1 - t0 - r));
+      TC_WAIT_WARP(FULL_C0 + s, (it >> 1) & 1, 18);
+      if (it >= 2) TC_WAIT_WARP(FC_FREE0 + s, ((it >> 1) - 1) & 1, 19);  // the MMA two blocks back has read this buffer
+      const __nv_bfloat16* ctile = &sm.st[s].c[0];
+      __nv_bfloat16* hi_tile = s ? sm.z_hi : sm.fc_hi;
+      __nv_bfloat16* lo_tile = s ? sm.z_lo : sm.fc_lo;
+#pragma unroll
+      for (int x2 = 0; x2 < 2; ++x2) {
+        const int off = r * 64 + (((2 * cq + x2) ^ (r & 7)) << 3);
+        const uint4 raw = *reinterpret_cast<const uint4*>(ctile + off);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        float x8[8];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[x]));
+          x8[2 * x] = v.x * f;
+          x8[2 * x + 1] = v.y * f;
+        }
+        uint4 h, l;
+        split8(x8, h, l);
+        *reinterpret_cast<uint4*>(hi_tile + off) = h;
+        if (split_c) *reinterpret_cast<uint4*>(lo_tile + off) = l;
+      }
+      fence_proxy_async_smem();
+      WARP_ARRIVE(FC_READY0 + s);
+      if (lane == 0) mbar_arrive(&sm.bars[C_FREE0 + s]);
+    }
+    if (warp >= 12) {
+      // segment-local state = accumulated dZ (hi-part + lo-part); this warp's 32 state columns of row r
+      const int zh = (warp - 12) >> 2;
+      const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+      TC_WAIT_WARP(DZ_READY, 0, 20);
+      tc_fence_after_sync();
+      float* dst = args.local_out + ((size_t)bh * args.nseg + seg) * (128 * 128) + (size_t)r * 128 + ehalf * 64 + zh * 32;
+#pragma unroll
+      for (int pc = 0; pc < 2; ++pc) {
+        uint32_t dh[16], dl[16];
+        tmem_ld_x16(lane_addr + COL_S0 + zh * 32 + pc * 16, dh);
+        if (split_c) tmem_ld_x16(lane_addr + COL_S0 + 64 + zh * 32 + pc * 16, dl);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          float4 v;
+          v.x = __uint_as_float(dh[4 * x]) + (split_c ? __uint_as_float(dl[4 * x]) : 0.f);
+          v.y = __uint_as_float(dh[4 * x + 1]) + (split_c ? __uint_as_float(dl[4 * x + 1]) : 0.f);
+          v.z = __uint_as_float(dh[4 * x + 2]) + (split_c ? __uint_as_float(dl[4 * x + 2]) : 0.f);
+          v.w = __uint_as_float(dh[4 * x + 3]) + (split_c ? __uint_as_float(dl[4 * x + 3]) : 0.f);
+          *reinterpret_cast<float4*>(dst + pc * 16 + 4 * x) = v;
+        }
+      }
+      tc_fence_before_sync();
+    }
   } else if (warp >= 4 && warp < 12) {
     // ------------------------------------ P group ------------------------------------
     if (!STATE_ONLY) {
@@ -496,7 +561,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       }
     }
   } else if (warp >= 12 && warp < 20) {
-    // ------------------------------------ Z group ------------------------------------
+    // ------------------------------------ Z group (walk kernel) ------------------------------------
     const int q = warp & 3;
     const int zh = (warp - 12) >> 2;  // which 32 of the 64 state / value columns this warp owns
     const int r = q * 32 + lane;      // token row j of c / state row k of Z
@@ -508,8 +573,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       const int t0 = seg_t0 + blk * 128;
       const int Cr = min(128, seg_t1 - t0);
       if (r >= Cr) return 0.f;
-      if (STATE_ONLY)
-        return REV ? exp2f(-s2 * (float)(t0 + r - seg_t0 + 1)) : exp2f(-s2 * (float)(seg_t1 - 1 - t0 - r));
       return REV ? exp2f(-s2 * (float)(r + 1)) : exp2f(-s2 * (float)(Cr - 1 - r));
     };
     // fc = diag(f_state) c for this warp's 32 columns of row r, given as 4 x 8 raw bf16 (chunks
@@ -533,14 +596,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       }
       fence_proxy_async_smem();
     };
-    // this thread's row slice of the c tile in shared memory (state-only kernel)
-    auto c_from_tile = [&](int it, uint4 (&raw)[4]) {
-      const __nv_bfloat16* ctile = &sm.st[it & 1].c[0];
-#pragma unroll
-      for (int x = 0; x < 4; ++x)
-        raw[x] = *reinterpret_cast<const uint4*>(ctile + r * 64 + (((4 * zh + x) ^ (r & 7)) << 3));
-    };
-    // the same slice straight from global memory (walk kernel: keeps the shared c tile off the state
+    // this thread's row slice of c straight from global memory (keeps the shared c tile off the state
     // chain, so that tile only has to arrive in time for M4); rows beyond N read as zero
     auto c_from_global = [&](int it, uint4 (&raw)[4]) {
       const int blk = REV ? (nblk - 1 - it) : it;
@@ -556,39 +612,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       }
     };
 
-    if (STATE_ONLY) {
-      for (int it = 0; it < nblk; ++it) {
-        const int s = it & 1;
-        TC_WAIT_WARP(FULL_C0 + s, (it >> 1) & 1, 18);
-        if (it >= 2) TC_WAIT_WARP(FC_FREE0 + s, ((it >> 1) - 1) & 1, 19);  // the MMA two blocks back has read this buffer
-        uint4 craw[4];
-        c_from_tile(it, craw);
-        make_fc(craw, state_factor(it), s ? sm.z_hi : sm.fc_hi, s ? sm.z_lo : sm.fc_lo);
-        WARP_ARRIVE(FC_READY0 + s);
-        if (lane == 0) mbar_arrive(&sm.bars[C_FREE0 + s]);
-      }
-      // segment-local state = accumulated dZ (hi-part + lo-part)
-      TC_WAIT_WARP(DZ_READY, 0, 20);
-      tc_fence_after_sync();
-      float* dst = args.local_out + ((size_t)bh * args.nseg + seg) * (128 * 128) + (size_t)r * 128 + ehalf * 64 + zh * 32;
-#pragma unroll
-      for (int pc = 0; pc < 2; ++pc) {
-        uint32_t dh[16], dl[16];
-        tmem_ld_x16(lane_addr + COL_S0 + zh * 32 + pc * 16, dh);
-        if (split_c) tmem_ld_x16(lane_addr + COL_S0 + 64 + zh * 32 + pc * 16, dl);
-        tmem_ld_wait();
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-          float4 v;
-          v.x = __uint_as_float(dh[4 * x]) + (split_c ? __uint_as_float(dl[4 * x]) : 0.f);
-          v.y = __uint_as_float(dh[4 * x + 1]) + (split_c ? __uint_as_float(dl[4 * x + 1]) : 0.f);
-          v.z = __uint_as_float(dh[4 * x + 2]) + (split_c ? __uint_as_float(dl[4 * x + 2]) : 0.f);
-          v.w = __uint_as_float(dh[4 * x + 3]) + (split_c ? __uint_as_float(dl[4 * x + 3]) : 0.f);
-          *reinterpret_cast<float4*>(dst + pc * 16 + 4 * x) = v;
-        }
-      }
-      tc_fence_before_sync();
-    } else {
+    {
       float zreg[32];
       if (args.entry) {
         const float4* src = reinterpret_cast<const float4*>(
