@@ -172,12 +172,20 @@ la_status la_fwd_noalloc(const la_shape* shape, const void* q, const void* k, co
  * Forward + backward with HOST tensors (end-to-end convenience; the paper has no
  * counterpart).  q,k,v,d_o and o,dq,dk,dv are host pointers with the layouts and
  * dtypes of la_fwd / la_bwd (pinned memory makes the copies asynchronous).  The
- * call enqueues, on `stream`: the four host-to-device copies, la_fwd, la_bwd
- * (zero initial state, no state gradients) and the four device-to-host copies.
- * device_arena is caller-owned device scratch of at least
+ * call enqueues the four host-to-device copies, la_fwd, la_bwd (zero initial
+ * state, no state gradients) and the four device-to-host copies.  Heads are
+ * independent, so for H >= 3 the work is cut into groups of heads that run as
+ * copy-in -> forward -> backward -> copy-out chains on three side streams owned
+ * by the library (created on first use, one set per device): copies of one
+ * group overlap the kernels and the opposite-direction copies of its
+ * neighbours.  The side streams start after all work queued on `stream` before
+ * the call, and `stream` continues only after they have finished, so to the
+ * caller the call behaves as if everything had been enqueued on `stream`.
+ * Calls from several host threads are enqueued one at a time and share the side
+ * streams, so they run one after the other on the device.  device_arena is caller-owned device scratch of at least
  * la_host_arena_bytes(shape) bytes, 256-byte aligned; it holds the device copies
- * of all eight tensors and the workspace.  Host outputs are valid once the
- * stream has been synchronised by the caller.
+ * of all eight tensors and the workspace.  Host outputs are valid once `stream`
+ * has been synchronised by the caller.
  */
 size_t la_host_arena_bytes(const la_shape* shape);
 la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void* k_host,

@@ -355,6 +355,37 @@ size_t la_host_arena_bytes(const la_shape* shape) {
   return total;
 }
 
+// Side streams and events of the host-buffer entry point: created once per device, on first use
+// (streams and events are not device memory; nothing here allocates any).
+namespace {
+constexpr int kHostLanes = 3;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t lane[kHostLanes];
+  cudaEvent_t done[kHostLanes];
+  cudaEvent_t start;
+};
+std::mutex g_pipe_mu;
+std::mutex g_pipe_enqueue_mu;  // one host thread at a time records and waits on the shared events
+HostPipe g_pipe[64];
+
+HostPipe* host_pipe() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_pipe_mu);
+  HostPipe& hp = g_pipe[dev];
+  if (!hp.ready) {
+    for (int i = 0; i < kHostLanes; ++i) {
+      if (cudaStreamCreateWithFlags(&hp.lane[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    if (cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    hp.ready = true;
+  }
+  return &hp;
+}
+}  // namespace
+
 la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void* k_host,
                           const void* v_host, const void* d_o_host, const float* lambda_host,
                           void* o_host, void* dq_host, void* dk_host, void* dv_host,
@@ -377,21 +408,86 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
   char* ws = p;
   const size_t ws_bytes = arena_bytes - (size_t)(ws - static_cast<char*>(device_arena));
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  LA_TRY_CUDA(cudaMemcpyAsync(dq_in, q_host, bq, cudaMemcpyHostToDevice, cs));
-  LA_TRY_CUDA(cudaMemcpyAsync(dk_in, k_host, bq, cudaMemcpyHostToDevice, cs));
-  LA_TRY_CUDA(cudaMemcpyAsync(dv_in, v_host, bv, cudaMemcpyHostToDevice, cs));
-  LA_TRY_CUDA(cudaMemcpyAsync(ddo_in, d_o_host, bv, cudaMemcpyHostToDevice, cs));
-  la_status st = la_fwd(shape, dq_in, dk_in, dv_in, lambda_host, d_o, nullptr, nullptr, ws, ws_bytes, stream);
-  if (st != LA_OK) return st;
-  // the forward workspace (first state set) feeds the backward pass, which uses the space behind it
-  const size_t wf = round256(la_workspace_bytes(LA_OP_FWD, shape));
-  st = la_bwd_reuse(shape, dq_in, dk_in, dv_in, ddo_in, lambda_host, d_dq, d_dk, d_dv, nullptr, nullptr, nullptr,
-                    wf > 0 ? ws : nullptr, ws + wf, ws_bytes - wf, stream);
-  if (st != LA_OK) return st;
-  LA_TRY_CUDA(cudaMemcpyAsync(o_host, d_o, bdv, cudaMemcpyDeviceToHost, cs));
-  LA_TRY_CUDA(cudaMemcpyAsync(dq_host, d_dq, bdq, cudaMemcpyDeviceToHost, cs));
-  LA_TRY_CUDA(cudaMemcpyAsync(dk_host, d_dk, bdq, cudaMemcpyDeviceToHost, cs));
-  LA_TRY_CUDA(cudaMemcpyAsync(dv_host, d_dv, bdv, cudaMemcpyDeviceToHost, cs));
+
+  // Heads are independent, so the work is cut into groups of heads that run as
+  // copy-in -> forward -> backward -> copy-out chains on three side streams: while one group
+  // computes, the next one's inputs arrive and the previous one's results leave, and the two copy
+  // directions share the link in full duplex.  Every group keeps the segment length of the whole
+  // shape, so its workspace is its heads' share of the whole workspace; the three streams use
+  // three disjoint thirds of it.
+  la_shape sub = *shape;
+  sub.B = 1;
+  sub.seg_len = la_segment_length(shape);
+  int group = shape->H / 8;
+  if (group < 1) group = 1;
+  size_t slot = 0;
+  HostPipe* hp = nullptr;
+  if (shape->H >= 3 * group) {
+    sub.H = group;
+    const size_t wf_g = la_workspace_bytes(LA_OP_FWD, &sub), wb_g = la_workspace_bytes(LA_OP_BWD, &sub);
+    if (wf_g != (size_t)-1 && wb_g != (size_t)-1) {
+      slot = round256(wf_g) + round256(wb_g);
+      if (slot * kHostLanes <= ws_bytes) hp = host_pipe();
+    }
+  }
+  if (!hp) {
+    // small shapes: one chain on the caller's stream
+    LA_TRY_CUDA(cudaMemcpyAsync(dq_in, q_host, bq, cudaMemcpyHostToDevice, cs));
+    LA_TRY_CUDA(cudaMemcpyAsync(dk_in, k_host, bq, cudaMemcpyHostToDevice, cs));
+    LA_TRY_CUDA(cudaMemcpyAsync(dv_in, v_host, bv, cudaMemcpyHostToDevice, cs));
+    LA_TRY_CUDA(cudaMemcpyAsync(ddo_in, d_o_host, bv, cudaMemcpyHostToDevice, cs));
+    la_status st = la_fwd(shape, dq_in, dk_in, dv_in, lambda_host, d_o, nullptr, nullptr, ws, ws_bytes, stream);
+    if (st != LA_OK) return st;
+    // the forward workspace (first state set) feeds the backward pass, which uses the space behind it
+    const size_t wf = round256(la_workspace_bytes(LA_OP_FWD, shape));
+    st = la_bwd_reuse(shape, dq_in, dk_in, dv_in, ddo_in, lambda_host, d_dq, d_dk, d_dv, nullptr, nullptr, nullptr,
+                      wf > 0 ? ws : nullptr, ws + wf, ws_bytes - wf, stream);
+    if (st != LA_OK) return st;
+    LA_TRY_CUDA(cudaMemcpyAsync(o_host, d_o, bdv, cudaMemcpyDeviceToHost, cs));
+    LA_TRY_CUDA(cudaMemcpyAsync(dq_host, d_dq, bdq, cudaMemcpyDeviceToHost, cs));
+    LA_TRY_CUDA(cudaMemcpyAsync(dk_host, d_dk, bdq, cudaMemcpyDeviceToHost, cs));
+    LA_TRY_CUDA(cudaMemcpyAsync(dv_host, d_dv, bdv, cudaMemcpyDeviceToHost, cs));
+    return LA_OK;
+  }
+
+  // the side streams start after everything already queued on the caller's stream ...
+  std::lock_guard<std::mutex> enqueue_lock(g_pipe_enqueue_mu);
+  LA_TRY_CUDA(cudaEventRecord(hp->start, cs));
+  for (int i = 0; i < kHostLanes; ++i) LA_TRY_CUDA(cudaStreamWaitEvent(hp->lane[i], hp->start, 0));
+  int g = 0;
+  for (int b = 0; b < shape->B; ++b) {
+    for (int h0 = 0; h0 < shape->H; h0 += group, ++g) {
+      const int hc = shape->H - h0 < group ? shape->H - h0 : group;
+      sub.H = hc;
+      cudaStream_t ls = hp->lane[g % kHostLanes];
+      char* wsg = ws + (size_t)(g % kHostLanes) * slot;
+      const size_t head = (size_t)b * shape->H + h0;  // first (b,h) slice of the group
+      const size_t oq = head * shape->N * shape->d * in_sz, ov = head * shape->N * shape->e * in_sz;
+      const size_t odq = head * shape->N * shape->d * out_sz, odv = head * shape->N * shape->e * out_sz;
+      const size_t nq = (size_t)hc * shape->N * shape->d * in_sz, nv = (size_t)hc * shape->N * shape->e * in_sz;
+      const size_t ndq = (size_t)hc * shape->N * shape->d * out_sz, ndv = (size_t)hc * shape->N * shape->e * out_sz;
+      LA_TRY_CUDA(cudaMemcpyAsync(dq_in + oq, static_cast<const char*>(q_host) + oq, nq, cudaMemcpyHostToDevice, ls));
+      LA_TRY_CUDA(cudaMemcpyAsync(dk_in + oq, static_cast<const char*>(k_host) + oq, nq, cudaMemcpyHostToDevice, ls));
+      LA_TRY_CUDA(cudaMemcpyAsync(dv_in + ov, static_cast<const char*>(v_host) + ov, nv, cudaMemcpyHostToDevice, ls));
+      LA_TRY_CUDA(cudaMemcpyAsync(ddo_in + ov, static_cast<const char*>(d_o_host) + ov, nv, cudaMemcpyHostToDevice, ls));
+      const size_t wf = round256(la_workspace_bytes(LA_OP_FWD, &sub));
+      la_status st = la_fwd(&sub, dq_in + oq, dk_in + oq, dv_in + ov, lambda_host + h0, d_o + odv, nullptr, nullptr,
+                            wsg, slot, ls);
+      if (st != LA_OK) return st;
+      st = la_bwd_reuse(&sub, dq_in + oq, dk_in + oq, dv_in + ov, ddo_in + ov, lambda_host + h0, d_dq + odq, d_dk + odq,
+                        d_dv + odv, nullptr, nullptr, nullptr, wf > 0 ? wsg : nullptr, wsg + wf, slot - wf, ls);
+      if (st != LA_OK) return st;
+      LA_TRY_CUDA(cudaMemcpyAsync(static_cast<char*>(o_host) + odv, d_o + odv, ndv, cudaMemcpyDeviceToHost, ls));
+      LA_TRY_CUDA(cudaMemcpyAsync(static_cast<char*>(dq_host) + odq, d_dq + odq, ndq, cudaMemcpyDeviceToHost, ls));
+      LA_TRY_CUDA(cudaMemcpyAsync(static_cast<char*>(dk_host) + odq, d_dk + odq, ndq, cudaMemcpyDeviceToHost, ls));
+      LA_TRY_CUDA(cudaMemcpyAsync(static_cast<char*>(dv_host) + odv, d_dv + odv, ndv, cudaMemcpyDeviceToHost, ls));
+    }
+  }
+  // ... and the caller's stream continues after all of them
+  for (int i = 0; i < kHostLanes; ++i) {
+    LA_TRY_CUDA(cudaEventRecord(hp->done[i], hp->lane[i]));
+    LA_TRY_CUDA(cudaStreamWaitEvent(cs, hp->done[i], 0));
+  }
   return LA_OK;
 }
 

@@ -417,3 +417,40 @@ def test_backward_reusing_forward_segment_states(path):
     tol = TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4
     for n, g, r in zip(("o", "dq", "dk", "dv", "grad_kv_in"), (o, dq, dk, dv, gin), (ref[0], ref[2], ref[3], ref[4], ref[5])):
         assert_close(g, r, tol, n)
+
+
+@pytest.mark.parametrize("B,H,N,seg_len", [(2, 8, 700, 0), (1, 5, 2100, 512), (1, 2, 900, 256)])
+def test_host_buffer_entry_point(B, H, N, seg_len):
+    """la_fwd_bwd_host: pinned host tensors in and out.  With H >= 3 the call pipelines groups of heads
+    over its side streams (the second case has a ragged last group and several segments per head), with
+    H < 3 it is a single chain; both must give exactly what la_fwd / la_bwd give on device tensors, and
+    that must agree with the oracle."""
+    d = 128
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=23)
+    lam = inputs.decay_rates(8, 0.5)[:H].contiguous()
+    shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, seg_len)
+    pin = lambda t: t.pin_memory()
+    qh, kh, vh, doh = pin(q), pin(k), pin(v), pin(do)
+    outs = [torch.empty((B, H, N, d), dtype=torch.float32).pin_memory() for _ in range(4)]
+    arena = torch.empty(la.host_arena_bytes(shape), dtype=torch.uint8, device=DEV)
+    for _ in range(2):  # the second call reuses the side streams
+        for t in outs:
+            t.fill_(float("nan"))
+        la.la_fwd_bwd_host(shape, qh, kh, vh, doh, lam, *outs, arena)
+        torch.cuda.synchronize()
+        la.device_status()
+        # the same on device tensors, with the backward pass reusing the forward pass's segment states as
+        # the host entry point does
+        qg, kg, vg, dog = to_dev(q, k, v, do)
+        dshape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, la.segment_length(shape))
+        o, dq, dk, dv = (torch.empty((B, H, N, d), dtype=torch.float32, device=DEV) for _ in range(4))
+        ws_f = la.alloc_workspace(la.LA_OP_FWD, dshape, DEV)
+        ws_b = la.alloc_workspace(la.LA_OP_BWD, dshape, DEV)
+        la.la_fwd(dshape, qg, kg, vg, lam, o, None, None, ws_f)
+        la.la_bwd(dshape, qg, kg, vg, dog, lam, dq, dk, dv, None, None, None, ws_b, fwd_workspace=ws_f)
+        torch.cuda.synchronize()
+        for n, h, g in zip(("o", "dq", "dk", "dv"), outs, (o, dq, dk, dv)):
+            assert torch.equal(h, g.cpu()), n
+    ref = oracle_all(q, k, v, do, lam, None, None)
+    for n, h, r in zip(("o", "dq", "dk", "dv"), outs, (ref[0], ref[2], ref[3], ref[4])):
+        assert_close(h, r, TOL_BF16, n)
