@@ -55,17 +55,6 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
       : "memory");
   return ok != 0;
 }
-// Bounded wait: returns false if the phase did not complete within ~budget clocks.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
-                                          long long budget = 4000000000LL) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > budget) return false;
-  }
-  return true;
-}
-
 // ---- proxy / tcgen05 fences -------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -178,18 +167,6 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 }
 
 // ---- TMEM loads: 32 lanes x 32-bit, N consecutive columns per thread ------------------------------
-__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -201,15 +178,7 @@ __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// ---- TMEM stores: 32 lanes x 32-bit, 16 consecutive columns per thread ---------------------------
-__device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
+// ---- TMEM stores: 32 lanes x 32-bit, 8 consecutive columns per thread ---------------------------
 __device__ __forceinline__ void tmem_st_x8(uint32_t taddr, const uint32_t (&r)[8]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
                "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
@@ -230,11 +199,11 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
 }
 
 // ---- warp-convergent issue -------------------------------------------------------------------------
-// The MMA-issuing warp runs its whole loop with all 32 lanes converged and only predicates the
-// tcgen05 instructions themselves on one elected lane.  Measured on B200: issued from inside a
-// divergent `if (lane == 0)` region, an MMA costs the issuing warp enough instruction slots that
-// arithmetic-heavy warps on the same scheduler stretch it from 48 to 122 clocks per instruction;
-// issued convergently (operands stay warp-uniform) it stays at the tensor pipe's own 46 clocks.
+// Used by the state-only kernel: the MMA-issuing warp runs its whole loop with all 32 lanes converged and
+// only predicates the tcgen05 instructions themselves on one elected lane.  Measured on B200 in a
+// micro-benchmark: issued from inside a divergent `if (lane == 0)` region, an MMA costs the issuing warp
+// enough instruction slots that FMA-bound warps on the same scheduler stretch it from 48 to 122 clocks
+// per instruction; issued convergently it stays at the tensor pipe's own 46 clocks.
 __device__ __forceinline__ uint32_t elect_one() {
   uint32_t el;
   asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(el));
@@ -252,18 +221,6 @@ __device__ __forceinline__ void umma_bf16_lh(uint32_t d_tmem, uint32_t a_lo, uin
       "mov.b64 db, {%2, %3};\n\t"
       "@g tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
       "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(go)
-      : "memory");
-}
-// Same with A in tensor memory.
-__device__ __forceinline__ void umma_bf16_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
-                                                uint32_t idesc, uint32_t accumulate, uint32_t go) {
-  asm volatile(
-      "{\n\t.reg .pred p, g;\n\t.reg .b64 db;\n\t"
-      "setp.ne.b32 g, %6, 0;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "@g tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(go)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit_if(uint64_t* bar, uint32_t go) {
