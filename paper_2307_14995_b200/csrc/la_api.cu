@@ -70,7 +70,7 @@ la_status check_shape(const la_shape* s, bool need_n) {
 }
 
 bool tensor_path_available(const la_shape* s) {
-  return tc_supported() && s->in_dtype == LA_BF16 && s->d == 128 && s->e == 128;
+  return tc_supported() && s->in_dtype == LA_BF16 && s->d == s->e && (s->d == 128 || s->d == 64);
 }
 
 la_status make_plan(const la_shape* s, Plan* p) {
@@ -86,7 +86,7 @@ la_status make_plan(const la_shape* s, Plan* p) {
     // time: pick the segment count that minimises (waves over the 148 SMs) x (blocks walked per
     // segment + pipeline fill), with segments no shorter than 1024 tokens so that the
     // per-segment state traffic stays small.  Depends on the shape only.
-    const long slices = p->tensor ? 2 : 1;  // the tensor kernels also split the value columns
+    const long slices = (p->tensor && s->d == 128) ? 2 : 1;  // at d = 128 the tensor kernels also split the value columns
     const long sms = 148, fill = 2;
     long most = s->N / 1024;
     if (most < 1) most = 1;
@@ -163,7 +163,7 @@ cudaError_t run_prepass(const la_shape* s, const Plan& p, const DecayTable& tab,
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
-  if (p.tensor) return launch_tc_prepass(args, tab, p.precision, st);
+  if (p.tensor) return launch_tc_prepass(args, tab, s->d, p.precision, st);
   return launch_simt_prepass(args, tab, s->d, s->e, (int)s->in_dtype, st);
 }
 
@@ -201,7 +201,7 @@ cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, co
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
-  if (p.tensor) return launch_tc_walk(args, tab, (int)s->out_dtype, p.precision, st);
+  if (p.tensor) return launch_tc_walk(args, tab, s->d, (int)s->out_dtype, p.precision, st);
   return launch_simt_walk(args, tab, s->d, s->e, (int)s->in_dtype, (int)s->out_dtype, st);
 }
 

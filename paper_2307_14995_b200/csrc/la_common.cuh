@@ -73,11 +73,11 @@ cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv
                           int H, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
                           cudaStream_t stream);
 
-// Tensor-core (tcgen05) kernels: bf16 inputs, Da = Ec = 128.
+// Tensor-core (tcgen05) kernels: bf16 inputs, Da = Ec = D with D = 64 or 128.
 bool tc_supported();
-cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int out_dt, int precision,
+cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int out_dt, int precision,
                            cudaStream_t stream);
-cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int precision,
+cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, int precision,
                               cudaStream_t stream);
 
 // Failure code recorded by a tensor-core block whose bounded wait expired (0 = none);

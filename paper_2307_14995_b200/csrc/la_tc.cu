@@ -216,7 +216,7 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     if (lane == 0) mbar_arrive(&sm.bars[barid]);         \
   } while (0)
 
-template <bool REV, bool STATE_ONLY, typename TOut>
+template <bool REV, bool STATE_ONLY, typename TOut, int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
           const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_out, const TcArgs args,
@@ -230,8 +230,14 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 #ifdef LA_TC_TRACE
   long long* const trace_ptr = (blockIdx.x == g_tc_trace_block) ? g_tc_trace : nullptr;
 #endif
-  const int ehalf = blockIdx.x & 1;
-  const int segid = blockIdx.x >> 1;
+  // D = 128: two thread blocks per (head, segment), one per half of the value columns.  D = 64: one
+  // thread block; the feature halves 64..127 of the a and b tiles do not exist (the K steps over them are
+  // skipped, and the second b panel, which M3 reads as rows 64..127 of b^T, is zeroed once below), so rows
+  // 64..127 of the state stay zero and are neither loaded nor stored.
+  static_assert(D == 64 || D == 128, "feature dimension");
+  constexpr int KD = D / 16;  // K steps over the feature dimension
+  const int ehalf = (D == 128) ? (int)(blockIdx.x & 1) : 0;
+  const int segid = (D == 128) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int bh = segid / args.nseg, seg = segid % args.nseg;
   const int seg_t0 = seg * args.seg_len;
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
@@ -264,6 +270,11 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     tmem_alloc(&sm.tmem_slot, TMEM_COLS);
     tmem_relinquish();
   }
+  if (D == 64) {
+    for (int i = tid; i < 2 * 1024; i += TC_THREADS)
+      reinterpret_cast<uint4*>(&sm.st[i >> 10].b[1][0])[i & 1023] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
+  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -288,20 +299,20 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         if (STATE_ONLY && it + 2 < nblk) {
           const int tp = seg_t0 + (REV ? (nblk - 3 - it) : (it + 2)) * 128;
           tma_prefetch_3d(&tm_b, 0, tp, bh);
-          tma_prefetch_3d(&tm_b, 64, tp, bh);
+          if (D == 128) tma_prefetch_3d(&tm_b, 64, tp, bh);
           tma_prefetch_3d(&tm_c, ehalf * 64, tp, bh);
         }
         if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
-        mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], 32768);
+        mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 256);
         tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
-        tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+        if (D == 128) tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
         armed_b[s] = (it >> 1) + 1;
         TC_TRACE(it, 0);
         if (!STATE_ONLY) {
           if (it >= 2) TC_WAIT(A_FREE0 + s, prev, 3);
-          mbar_arrive_expect_tx(&sm.bars[FULL_A0 + s], 32768);
+          mbar_arrive_expect_tx(&sm.bars[FULL_A0 + s], D * 256);
           tma_load_3d(&stg.a[0][0], &tm_a, &sm.bars[FULL_A0 + s], 0, t0, bh);
-          tma_load_3d(&stg.a[1][0], &tm_a, &sm.bars[FULL_A0 + s], 64, t0, bh);
+          if (D == 128) tma_load_3d(&stg.a[1][0], &tm_a, &sm.bars[FULL_A0 + s], 64, t0, bh);
           armed_a[s] = (it >> 1) + 1;
           TC_TRACE(it, 2);
         }
@@ -364,7 +375,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           TC_WAIT(FULL_B0, 0, 7);
           tc_fence_after_sync();
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
+          for (int k = 0; k < KD; ++k) {
             const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
             umma_bf16(tmem + COL_S0, umma_desc_sw128(a0 + ko, 16, 1024), umma_desc_sw128(b0 + ko, 16, 1024), ID_S,
                       k > 0);
@@ -404,14 +415,14 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           tc_fence_after_sync();
           TC_TRACE(it, 5);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
+          for (int k = 0; k < KD; ++k) {
             const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
             umma_bf16(tmem + col_oe, umma_desc_sw128(a0 + ko, 16, 1024),
                       umma_desc_sw128(zh0 + k * 2048, 16384, 1024), ID_KN, k > 0);
           }
           if (split_z) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < KD; ++k) {
               const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
               umma_bf16(tmem + col_oe, umma_desc_sw128(a0 + ko, 16, 1024),
                         umma_desc_sw128(zl0 + k * 2048, 16384, 1024), ID_KN, 1);
@@ -430,7 +441,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             tc_fence_after_sync();
             TC_TRACE(it, 4);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < KD; ++k) {
               const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
               umma_bf16(tmem + (s1 ? COL_S1 : COL_S0), umma_desc_sw128(an + ko, 16, 1024),
                         umma_desc_sw128(bn + ko, 16, 1024), ID_S, k > 0);
@@ -505,9 +516,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
       TC_WAIT_WARP(DZ_READY, 0, 20);
       tc_fence_after_sync();
-      float* dst = args.local_out + ((size_t)bh * args.nseg + seg) * (128 * 128) + (size_t)r * 128 + ehalf * 64 + zh * 32;
+      float* dst = args.local_out + ((size_t)bh * args.nseg + seg) * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32;
 #pragma unroll
       for (int pc = 0; pc < 2; ++pc) {
+        if (r >= D) break;  // D = 64: state rows 64..127 do not exist (warp-uniform: r = 32 q + lane)
         uint32_t dh[16], dl[16];
         tmem_ld_x16(lane_addr + COL_S0 + zh * 32 + pc * 16, dh);
         if (split_c) tmem_ld_x16(lane_addr + COL_S0 + 64 + zh * 32 + pc * 16, dl);
@@ -619,7 +631,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       const int t = seg_t0 + blk * 128 + r;
       if (t < args.N) {
         const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(args.c) +
-                                                          ((size_t)bh * args.N + t) * 128 + ehalf * 64 + zh * 32);
+                                                          ((size_t)bh * args.N + t) * D + ehalf * 64 + zh * 32);
 #pragma unroll
         for (int x = 0; x < 4; ++x) raw[x] = __ldg(src + x);
       } else {
@@ -630,9 +642,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 
     {
       float zreg[32];
-      if (args.entry) {
+      if (args.entry && r < D) {
         const float4* src = reinterpret_cast<const float4*>(
-            args.entry + ((size_t)bh * args.nseg + seg) * (128 * 128) + (size_t)r * 128 + ehalf * 64 + zh * 32);
+            args.entry + ((size_t)bh * args.nseg + seg) * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32);
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
           const float4 v = __ldg(src + x);
@@ -699,8 +711,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
       }
       const bool last_processed = REV ? (seg == 0) : (seg == args.nseg - 1);
-      if (args.final_out && last_processed) {
-        float* dst = args.final_out + (size_t)bh * (128 * 128) + (size_t)r * 128 + ehalf * 64 + zh * 32;
+      if (args.final_out && last_processed && r < D) {
+        float* dst = args.final_out + (size_t)bh * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32;
 #pragma unroll
         for (int x = 0; x < 8; ++x)
           *reinterpret_cast<float4*>(dst + 4 * x) = make_float4(zreg[4 * x], zreg[4 * x + 1], zreg[4 * x + 2], zreg[4 * x + 3]);
@@ -828,14 +840,14 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over a [BH, N, 128] tensor (feature dimension innermost) of bf16 or fp32 with a box of
+// Tensor map over a [BH, N, D] tensor (feature dimension innermost, D = 64 or 128) of bf16 or fp32 with a box of
 // 128 bytes x 128 rows x 1 and 128-byte swizzle; rows beyond N read as zero and are not written.
-bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, bool f32 = false) {
+bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, int D, bool f32 = false) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   const cuuint64_t esz = f32 ? 4 : 2;
-  cuuint64_t dims[3] = {128, (cuuint64_t)N, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {128 * esz, (cuuint64_t)N * 128 * esz};
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {D * esz, (cuuint64_t)N * D * esz};
   cuuint32_t box[3] = {(cuuint32_t)(128 / esz), 128, 1};
   cuuint32_t es[3] = {1, 1, 1};
   return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr),
@@ -843,46 +855,57 @@ bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, bool f32 = false) 
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool REV, bool STATE_ONLY, typename TOut>
+template <bool REV, bool STATE_ONLY, typename TOut, int D>
 cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mo,
                      const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
   const size_t smem = sizeof(TcSmem) + 1024;
-  auto kern = tc_kernel<REV, STATE_ONLY, TOut>;
+  auto kern = tc_kernel<REV, STATE_ONLY, TOut, D>;
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   KernelTimer timer(STATE_ONLY ? K_PREPASS : K_WALK, stream);
-  kern<<<(unsigned)(ta.BH * ta.nseg * 2), TC_THREADS, smem, stream>>>(ma, mb, mc, mo, ta, tab);
+  kern<<<(unsigned)(ta.BH * ta.nseg * (D == 128 ? 2 : 1)), TC_THREADS, smem, stream>>>(ma, mb, mc, mo, ta, tab);
   count_launch();
   return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_walk_d(const OpArgs& args, const DecayTable& tab, int out_dt, int precision, cudaStream_t stream) {
+  CUtensorMap ma, mb, mc, mo;
+  const bool f32 = (out_dt == DT_F32);
+  if (!make_map(&ma, args.a, args.N, args.BH, D) || !make_map(&mb, args.b, args.N, args.BH, D) ||
+      !make_map(&mc, args.c, args.N, args.BH, D) || !make_map(&mo, args.out, args.N, args.BH, D, f32))
+    return cudaErrorInvalidValue;
+  TcArgs ta{args.c, args.out, args.entry, nullptr, args.final_out, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
+  if (args.reverse)
+    return f32 ? launch_t<true, false, float, D>(ma, mb, mc, mo, ta, tab, stream)
+               : launch_t<true, false, __nv_bfloat16, D>(ma, mb, mc, mo, ta, tab, stream);
+  return f32 ? launch_t<false, false, float, D>(ma, mb, mc, mo, ta, tab, stream)
+             : launch_t<false, false, __nv_bfloat16, D>(ma, mb, mc, mo, ta, tab, stream);
+}
+
+template <int D>
+cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int precision, cudaStream_t stream) {
+  CUtensorMap mb, mc;
+  if (!make_map(&mb, args.b, args.N, args.BH, D) || !make_map(&mc, args.c, args.N, args.BH, D))
+    return cudaErrorInvalidValue;
+  TcArgs ta{args.c, nullptr, nullptr, args.local_out, nullptr, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
+  // the a and out maps are unused by the state-only kernel; pass valid descriptors anyway
+  return args.reverse ? launch_t<true, true, float, D>(mb, mb, mc, mc, ta, tab, stream)
+                      : launch_t<false, true, float, D>(mb, mb, mc, mc, ta, tab, stream);
 }
 
 }  // namespace
 
 bool tc_supported() { return encode_fn() != nullptr; }
 
-cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int out_dt, int precision,
+cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int out_dt, int precision,
                            cudaStream_t stream) {
-  CUtensorMap ma, mb, mc, mo;
-  const bool f32 = (out_dt == DT_F32);
-  if (!make_map(&ma, args.a, args.N, args.BH) || !make_map(&mb, args.b, args.N, args.BH) ||
-      !make_map(&mc, args.c, args.N, args.BH) || !make_map(&mo, args.out, args.N, args.BH, f32))
-    return cudaErrorInvalidValue;
-  TcArgs ta{args.c, args.out, args.entry, nullptr, args.final_out, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
-  if (args.reverse)
-    return f32 ? launch_t<true, false, float>(ma, mb, mc, mo, ta, tab, stream)
-               : launch_t<true, false, __nv_bfloat16>(ma, mb, mc, mo, ta, tab, stream);
-  return f32 ? launch_t<false, false, float>(ma, mb, mc, mo, ta, tab, stream)
-             : launch_t<false, false, __nv_bfloat16>(ma, mb, mc, mo, ta, tab, stream);
+  return D == 128 ? launch_walk_d<128>(args, tab, out_dt, precision, stream)
+                  : launch_walk_d<64>(args, tab, out_dt, precision, stream);
 }
 
-cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int precision, cudaStream_t stream) {
-  CUtensorMap mb, mc;
-  if (!make_map(&mb, args.b, args.N, args.BH) || !make_map(&mc, args.c, args.N, args.BH))
-    return cudaErrorInvalidValue;
-  TcArgs ta{args.c, nullptr, nullptr, args.local_out, nullptr, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
-  // the a and out maps are unused by the state-only kernel; pass valid descriptors anyway
-  return args.reverse ? launch_t<true, true, float>(mb, mb, mc, mc, ta, tab, stream)
-                      : launch_t<false, true, float>(mb, mb, mc, mc, ta, tab, stream);
+cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, int precision, cudaStream_t stream) {
+  return D == 128 ? launch_prepass_d<128>(args, tab, precision, stream) : launch_prepass_d<64>(args, tab, precision, stream);
 }
 
 #ifdef LA_TC_TRACE
