@@ -377,7 +377,7 @@ def run_ours(args):
                         "tflops": world * ow.token_heads * oF / (oms * 1e-3) / 1e12,
                         "tokens_per_s": world * ow.B * ow.N / (oms * 1e-3),
                         "step_roofline_frac": oroof * 1e3 / oms, "l2": "flushed between timed steps",
-                        "kernels": "tcgen05" if ow.d == 128 else "fp32 CUDA cores (d = 64)"}
+                        "kernels": "tcgen05 (one thread block per head and segment at d = 64, two at d = 128)"}
         del od_, oo, odq, odk, odv, owf, owb, flush
 
     clocks = sampler.stop() if rank == 0 else None
