@@ -68,7 +68,7 @@ enum Bar {
   A_FREE0, A_FREE1, B_FREE0, B_FREE1, C_FREE0, C_FREE1,       // consumers -> TMA
   S_READY0, S_READY1, P_READY0, P_READY1,
   FC_READY0, FC_READY1, FC_FREE0, FC_FREE1,                   // (second buffer: state-only kernel)
-  DZ_READY, DZ_FREE, Z_READY, Z_FREE, O_READY, O_FREE, OG_SYNC, DRAIN,
+  DZ_READY, Z_READY, O_READY, O_FREE, OG_SYNC, DRAIN,
   NUM_BARS
 };
 
@@ -252,7 +252,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     for (int i = 0; i < NUM_BARS; ++i) {
       uint32_t count = 1;
       // barriers that a compute group arrives on: one arrival per warp
-      if (i == P_READY0 || i == P_READY1 || i == FC_READY0 || i == FC_READY1 || i == Z_READY || i == DZ_FREE)
+      if (i == P_READY0 || i == P_READY1 || i == FC_READY0 || i == FC_READY1 || i == Z_READY)
         count = (STATE_ONLY && (i == FC_READY0 || i == FC_READY1)) ? 16 : 8;
       if (i == O_FREE || i == OG_SYNC) count = 4;
       // the c tile is released by the warps that read it (state-only) / by the thread that stores from it (walk)
@@ -302,20 +302,23 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           if (D == 128) tma_prefetch_3d(&tm_b, 64, tp, bh);
           tma_prefetch_3d(&tm_c, ehalf * 64, tp, bh);
         }
-        if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
-        mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 256);
-        tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
-        if (D == 128) tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+        if (STATE_ONLY) {
+          if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
+          mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 256);
+          tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
+          if (D == 128) tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+        } else {
+          // walk kernel: the a and b tiles of a stage travel together (one barrier for both, FULL_B); A_FREE
+          // is committed after M2, the last product of the block that reads either of them
+          if (it >= 2) TC_WAIT(A_FREE0 + s, prev, 3);
+          mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 512);
+          tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
+          if (D == 128) tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+          tma_load_3d(&stg.a[0][0], &tm_a, &sm.bars[FULL_B0 + s], 0, t0, bh);
+          if (D == 128) tma_load_3d(&stg.a[1][0], &tm_a, &sm.bars[FULL_B0 + s], 64, t0, bh);
+        }
         armed_b[s] = (it >> 1) + 1;
         TC_TRACE(it, 0);
-        if (!STATE_ONLY) {
-          if (it >= 2) TC_WAIT(A_FREE0 + s, prev, 3);
-          mbar_arrive_expect_tx(&sm.bars[FULL_A0 + s], D * 256);
-          tma_load_3d(&stg.a[0][0], &tm_a, &sm.bars[FULL_A0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.a[1][0], &tm_a, &sm.bars[FULL_A0 + s], 64, t0, bh);
-          armed_a[s] = (it >> 1) + 1;
-          TC_TRACE(it, 2);
-        }
         if (it >= 2) TC_WAIT(C_FREE0 + s, prev, 2);
         mbar_arrive_expect_tx(&sm.bars[FULL_C0 + s], 16384);
         tma_load_3d(&stg.c[0], &tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, bh);
@@ -371,8 +374,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         // prologue: S(0)
         {
           const uint32_t a0 = smem_u32(&sm.st[0].a[0][0]), b0 = smem_u32(&sm.st[0].b[0][0]);
-          TC_WAIT(FULL_A0, 0, 6);
-          TC_WAIT(FULL_B0, 0, 7);
+          TC_WAIT(FULL_B0, 0, 7);  // a and b of block 0
           tc_fence_after_sync();
 #pragma unroll
           for (int k = 0; k < KD; ++k) {
@@ -391,8 +393,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           const uint32_t col_p = s ? COL_S1 : COL_S0;
           // M3: dZ = b^T [fc_hi | fc_lo]  (needs the previous dZ to have been read)
           TC_TRACE(it, 15);
-          TC_WAIT(FC_READY0, par1, 8);
-          if (it > 0) TC_WAIT(DZ_FREE, (it - 1) & 1, 9);
+          // Z_READY: the state operand of this block AND fc of this block are in place (the Z group forms fc first)
+          TC_WAIT(Z_READY, par1, 12);
           tc_fence_after_sync();
           TC_TRACE(it, 3);
 #pragma unroll
@@ -406,10 +408,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                         umma_desc_sw128(fh0 + 16384 + k * 2048, 16384, 1024), ID_MN64, 1);
           }
           umma_commit(&sm.bars[DZ_READY]);
-          umma_commit(&sm.bars[B_FREE0 + s]);
           TC_TRACE(it, 16);
           // M2: O_inter = a Z   (state after the previous block / the entry state)
-          TC_WAIT(Z_READY, par1, 12);
           // this O_inter buffer was last read for block it-2; that read was already awaited before M4(it-1)
           const uint32_t col_oe = (it & 1) ? COL_OE1 : COL_OE0;
           tc_fence_after_sync();
@@ -428,7 +428,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                         umma_desc_sw128(zl0 + k * 2048, 16384, 1024), ID_KN, 1);
             }
           }
-          umma_commit(&sm.bars[Z_FREE]);
           umma_commit(&sm.bars[A_FREE0 + s]);  // M1 and M2 of this block are done with the a tile
           TC_TRACE(it, 19);
           // M1 of the next block, into the other S/P buffer
@@ -436,8 +435,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             const int s1 = s ^ 1;
             const uint32_t parn = ((it + 1) >> 1) & 1;
             const uint32_t an = smem_u32(&sm.st[s1].a[0][0]), bn = smem_u32(&sm.st[s1].b[0][0]);
-            TC_WAIT(FULL_A0 + s1, parn, 10);
-            TC_WAIT(FULL_B0 + s1, parn, 11);
+            TC_WAIT(FULL_B0 + s1, parn, 11);  // a and b of the next block
             tc_fence_after_sync();
             TC_TRACE(it, 4);
 #pragma unroll
@@ -669,13 +667,12 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
         fence_proxy_async_smem();
       };
-      write_state_operand();
-      WARP_ARRIVE(Z_READY);
       uint4 cnext[4];  // row slice of the next block's c, fetched one block ahead
       c_from_global(0, cnext);
       make_fc(cnext, state_factor(0), sm.fc_hi, sm.fc_lo);
-      WARP_ARRIVE(FC_READY0);
       if (nblk > 1) c_from_global(1, cnext);
+      write_state_operand();
+      WARP_ARRIVE(Z_READY);
 
       for (int it = 0; it < nblk; ++it) {
         const int blk = REV ? (nblk - 1 - it) : it;
@@ -694,17 +691,15 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 #pragma unroll
             for (int x = 0; x < 16; ++x) zreg[pc * 16 + x] = fmaf(gamma, zreg[pc * 16 + x], __uint_as_float(dh[x]));
           }
-          tc_fence_before_sync();
-          WARP_ARRIVE(DZ_FREE);
+          tc_fence_before_sync();  // ordered before the Z_READY arrival below, which is what M3 of the next block waits for
         }
         if (it + 1 < nblk) {
           // DZ_READY also says M3 of this block is done, so the fc buffer may be rewritten
           make_fc(cnext, state_factor(it + 1), sm.fc_hi, sm.fc_lo);
-          WARP_ARRIVE(FC_READY0);
           if (it + 2 < nblk) c_from_global(it + 2, cnext);
           if (tid == 384) TC_TRACE(it, 10);
-          // Z_FREE: M2 of this block has read the old state operand
-          TC_WAIT_WARP(Z_FREE, it & 1, 23);
+          // A_FREE of this block's stage: M2 of this block is done, so it has read the old state operand
+          TC_WAIT_WARP(A_FREE0 + (it & 1), (it >> 1) & 1, 23);
           write_state_operand();
           WARP_ARRIVE(Z_READY);
           if (tid == 384) TC_TRACE(it, 11);
