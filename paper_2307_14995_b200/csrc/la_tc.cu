@@ -68,7 +68,7 @@ enum Bar {
   A_FREE0, A_FREE1, B_FREE0, B_FREE1, C_FREE0, C_FREE1,       // consumers -> TMA
   S_READY0, S_READY1, P_READY0, P_READY1,
   FC_READY0, FC_READY1, FC_FREE0, FC_FREE1,                   // (second buffer: state-only kernel)
-  DZ_READY, Z_READY, O_READY, O_FREE, OG_SYNC, DRAIN,
+  DZ_READY, Z_READY, O_READY, OG_SYNC, DRAIN,
   NUM_BARS
 };
 
@@ -254,7 +254,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       // barriers that a compute group arrives on: one arrival per warp
       if (i == P_READY0 || i == P_READY1 || i == FC_READY0 || i == FC_READY1 || i == Z_READY)
         count = (STATE_ONLY && (i == FC_READY0 || i == FC_READY1)) ? 16 : 8;
-      if (i == O_FREE || i == OG_SYNC) count = 4;
+      // P_READY of a block completes when the P group has written P AND the output group has read the
+      // previous block's accumulators (both are what M4 waits for): 8 + 4 warps
+      if (i == P_READY0 || i == P_READY1) count = 12;
+      if (i == OG_SYNC) count = 4;
       // the c tile is released by the warps that read it (state-only) / by the thread that stores from it (walk)
       if (i == C_FREE0 || i == C_FREE1) count = STATE_ONLY ? 16 : 1;
       mbar_init(&sm.bars[i], count);
@@ -448,9 +451,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           }
           // M4: O_intra = P c, P read from tensor memory (K step k: hi pairs at column 16k, lo pairs at 16k+8)
           TC_TRACE(it, 20);
-          TC_WAIT(P_READY0 + s, par2, 14);
+          TC_WAIT(P_READY0 + s, par2, 14);  // P is written and the accumulators of the previous block have been read
           TC_WAIT(FULL_C0 + s, par2, 15);
-          if (it > 0) TC_WAIT(O_FREE, (it - 1) & 1, 26);  // O_intra of the previous block has been read
           tc_fence_after_sync();
           TC_TRACE(it, 6);
 #pragma unroll
@@ -720,6 +722,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       const int r = q * 32 + lane;  // output row i
       const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
       uint32_t og_uses = 0;  // phases of the group's own barrier used so far
+      if (lane == 0) mbar_arrive(&sm.bars[P_READY0]);  // block 0 has no earlier accumulators to wait for
       for (int it = 0; it < nblk; ++it) {
         const int s = it & 1;
         const int blk = REV ? (nblk - 1 - it) : it;
@@ -747,7 +750,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             tmem_ld_wait();
             if (pass == PASSES - 1 && pc == PIECES - 1) {
               tc_fence_before_sync();
-              WARP_ARRIVE(O_FREE);  // both accumulators are in registers now
+              // both accumulators are in registers now: M4 of the next block may overwrite O_intra
+              if (it + 1 < nblk) WARP_ARRIVE(P_READY0 + (s ^ 1));
               if (tid == 736) TC_TRACE(it, 13);
             }
             if (sizeof(TOut) == 4) {
