@@ -1,5 +1,6 @@
 // Tensor-core kernels of the generic decayed linear-attention operator for
-// bf16 inputs with Da = Ec = 128 (block formulas: la_common.cuh).
+// bf16 inputs with Da = Ec = D, D = 128 or 64 (block formulas: la_common.cuh; the text below is for
+// D = 128, the differences at D = 64 are described at the kernel's template parameter).
 //
 // One thread block walks the 128-token blocks of one (batch*head, segment,
 // half of the value columns).  Per block it issues, on the 5th-generation
@@ -30,10 +31,16 @@
 //   warps 12-19  "Z" group (two warps per quarter, 32 state columns each): owns the fp32 state
 //                in registers (Z <- Gamma Z + dZ), rewrites the bf16 state operand, and forms
 //                fc = diag(f_state) c of the next block
-//   warps 20-23  "O" group: out = O_intra + diag(f_out) O_inter; rows pass through a per-warp
-//                scratch (the dead c tile) so that global stores cover whole 128-byte lines
+//   warps 20-23  "O" group: out = O_intra + diag(f_out) O_inter; 128 bytes of every output row are
+//                staged in the dead c tile and leave through bulk tensor stores
+// In the state-only pre-pass warps 4-19 all form fc, and the MMA warp issues converged.
 // All hand-offs are mbarriers; every wait is bounded and an expired wait makes the whole
-// block unwind (flag set, copies drained, tensor memory freed).
+// block unwind (flag set, copies drained, tensor memory freed).  Barrier operations on the MMA
+// lane are kept few, since each costs the lane about a hundred clocks (measured): per block it
+// waits for Z_READY (state operand and fc, both written by the Z group), FULL_B of the next block
+// (a and b tiles travel together), P_READY (P written AND the previous block's accumulators read
+// by the output group: 8 + 4 arrivals) and FULL_C, and commits to DZ_READY, A_FREE (which the
+// producer and the Z group both wait for), S_READY and O_READY.
 //
 // The only chain that is sequential across blocks is dZ -> Z -> O_inter; S, P and fc of
 // block n+1 do not depend on block n.  The MMA lane therefore issues, per block n:
@@ -64,7 +71,7 @@ constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_OI = 256, COL_OE0 = 320, COL_OE
 constexpr long long WAIT_BUDGET = 2000000000LL;  // clocks (~1 s)
 
 enum Bar {
-  FULL_A0 = 0, FULL_A1, FULL_B0, FULL_B1, FULL_C0, FULL_C1,   // TMA -> consumers
+  FULL_B0 = 0, FULL_B1, FULL_C0, FULL_C1,                     // TMA -> consumers (FULL_B: b, and a in the walk kernel)
   A_FREE0, A_FREE1, B_FREE0, B_FREE1, C_FREE0, C_FREE1,       // consumers -> TMA
   S_READY0, S_READY1, P_READY0, P_READY1,
   FC_READY0, FC_READY1, FC_FREE0, FC_FREE1,                   // (second buffer: state-only kernel)
@@ -285,7 +292,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   TC_CTA_TIME(0);
   bool issued_mma = false;
   uint32_t mma_elected = 0;  // set in the lane of warp 1 that issues the tensor-core instructions
-  int armed_a[2] = {0, 0}, armed_b[2] = {0, 0}, armed_c[2] = {0, 0};  // producer: uses armed per stage
+  int armed_b[2] = {0, 0}, armed_c[2] = {0, 0};  // producer: uses armed per stage
 
   if (warp == 0) {
     // ------------------------------------ TMA producer ------------------------------------
@@ -807,7 +814,6 @@ teardown:
   if (sm.abort) {
     if (warp == 0 && lane == 0) {
       for (int s = 0; s < 2; ++s) {
-        if (armed_a[s] > 0) drain_wait(&sm.bars[FULL_A0 + s], (armed_a[s] - 1) & 1);
         if (armed_b[s] > 0) drain_wait(&sm.bars[FULL_B0 + s], (armed_b[s] - 1) & 1);
         if (armed_c[s] > 0) drain_wait(&sm.bars[FULL_C0 + s], (armed_c[s] - 1) & 1);
       }
