@@ -203,6 +203,16 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
  */
 la_status la_device_status(unsigned int* code);
 
+/*
+ * Self-test of that failure path (no counterpart in the paper): launches one warp
+ * that waits, with the kernels' own bounded wait, on a barrier nothing ever arrives
+ * on.  After budget_clocks SM clocks (1 .. 2e9; 2e6 is about a millisecond) the
+ * wait gives up, records code 99 and the kernel returns normally; the next
+ * la_device_status() reports LA_ERR_DEVICE_TIMEOUT with that code and the context
+ * stays usable.  Nothing faults, traps or spins without limit.
+ */
+la_status la_selftest_bounded_wait(unsigned long long budget_clocks, void* stream);
+
 /* Human-readable name of a status code (static string). */
 const char* la_status_string(la_status s);
 

@@ -73,6 +73,8 @@ def load():
         lib.la_host_arena_bytes.restype = sz
         lib.la_fwd_bwd_host.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, sz, vp]
         lib.la_fwd_bwd_host.restype = I
+        lib.la_selftest_bounded_wait.argtypes = [ctypes.c_ulonglong, vp]
+        lib.la_selftest_bounded_wait.restype = I
         lib.la_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint)]
         lib.la_device_status.restype = I
         lib.la_status_string.argtypes = [I]
@@ -107,6 +109,13 @@ def device_status() -> int:
     if rc != 0:
         raise LaError(rc, "la_device_status (device code %d)" % code.value)
     return int(code.value)
+
+
+def selftest_bounded_wait(budget_clocks: int, stream=None) -> None:
+    """Launch the bounded-wait self-test (see la.h); the outcome is read with device_status()."""
+    rc = load().la_selftest_bounded_wait(int(budget_clocks), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_selftest_bounded_wait")
 
 
 def profile_enable(on: bool) -> None:

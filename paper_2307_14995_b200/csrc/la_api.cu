@@ -491,6 +491,15 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
   return LA_OK;
 }
 
+la_status la_selftest_bounded_wait(unsigned long long budget_clocks, void* stream) {
+  if (budget_clocks == 0 || budget_clocks > 2000000000ull) return LA_ERR_INVALID_ARG;
+  const la_status dev = check_device();
+  if (dev != LA_OK) return dev;
+  if (launch_bounded_wait_selftest((long long)budget_clocks, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return LA_ERR_CUDA;
+  return LA_OK;
+}
+
 la_status la_device_status(unsigned int* code) {
   if (cudaDeviceSynchronize() != cudaSuccess) return LA_ERR_CUDA;
   const unsigned int v = tc_read_status(true);

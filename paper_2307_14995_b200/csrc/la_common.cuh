@@ -80,6 +80,9 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int
 cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, int precision,
                               cudaStream_t stream);
 
+// One warp runs the kernels' bounded wait on a barrier nothing arrives on (budget in SM clocks).
+cudaError_t launch_bounded_wait_selftest(long long budget_clocks, cudaStream_t stream);
+
 // Failure code recorded by a tensor-core block whose bounded wait expired (0 = none);
 // copies it from the device (blocking) and optionally clears it.
 unsigned int tc_read_status(bool clear);

@@ -106,14 +106,15 @@ struct TcArgs {
   int precision;
 };
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                              long long budget = WAIT_BUDGET) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   // each try blocks in hardware for the default time limit (it returns early when the phase completes);
   // measured: giving a suspend-time hint of 1, 20 or 200 us instead makes the walk kernel 4 % slower
   while (!mbar_try_wait(bar, parity)) {
     if (*abort_flag) return false;
-    if (clock64() - t0 > WAIT_BUDGET) return false;
+    if (clock64() - t0 > budget) return false;
   }
   return true;
 }
@@ -829,6 +830,22 @@ teardown:
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
+// Self-test of the failure path: one warp waits, with the kernels' own bounded wait, on a barrier that
+// nothing ever arrives on; when the budget runs out it records code 99 like a real block would and returns.
+__global__ void bounded_wait_selftest_kernel(long long budget) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (!wait_or_abort(&bar, 0, &abort_flag, budget)) {
+    if (threadIdx.x == 0) atomicCAS(&g_tc_status, 0u, 99u);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -922,6 +939,12 @@ extern "C" void la_debug_set_cta_times(unsigned long long* device_buffer) {
   cudaMemcpyToSymbol(g_tc_cta_times, &device_buffer, sizeof(device_buffer));
 }
 #endif
+
+cudaError_t launch_bounded_wait_selftest(long long budget_clocks, cudaStream_t stream) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(budget_clocks);
+  count_launch();
+  return cudaGetLastError();
+}
 
 unsigned int tc_read_status(bool clear) {
   unsigned int v = 0;

@@ -454,3 +454,26 @@ def test_host_buffer_entry_point(B, H, N, seg_len):
     ref = oracle_all(q, k, v, do, lam, None, None)
     for n, h, r in zip(("o", "dq", "dk", "dv"), outs, (ref[0], ref[2], ref[3], ref[4])):
         assert_close(h, r, TOL_BF16, n)
+
+
+def test_bounded_wait_expires_cleanly():
+    """Failure path of the tensor-core kernels, exercised without any fault: a warp waits on a barrier
+    nothing arrives on, the wait gives up after its (here short) budget and records a code, the host reads
+    LA_ERR_DEVICE_TIMEOUT, the flag clears, and the context keeps working."""
+    la.device_status()                       # start from a clean flag
+    la.selftest_bounded_wait(2_000_000)      # about a millisecond
+    with pytest.raises(la.LaError) as ei:
+        la.device_status()
+    assert ei.value.code == 6                # LA_ERR_DEVICE_TIMEOUT
+    assert "device code 99" in str(ei.value)
+    assert la.device_status() == 0           # reading the flag cleared it
+    # the context is intact: a normal call still gives the right answer
+    q, k, v, _ = inputs.make_qkvdo(1, 2, 300, 128, 128, seed=3, with_do=False)
+    lam = torch.tensor([1.0, 0.9])
+    qg, kg, vg = to_dev(q, k, v)
+    o = la.fwd(qg, kg, vg, lam)
+    torch.cuda.synchronize()
+    la.device_status()
+    assert_close(o, orc.fwd_rec(q, k, v, lam.double().numpy()), TOL_BF16, "o")
+    with pytest.raises(la.LaError):
+        la.selftest_bounded_wait(0)          # budget out of range: refused before any launch
