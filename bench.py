@@ -276,6 +276,22 @@ def run_ours(args):
                               "walk_gbs": achieved}), flush=True)
         return
 
+    # forward and backward also timed on their own (same buffers, same rules), after the headline loop
+    split_ms = {}
+    for nm, fn in (("fwd", lambda: la.la_fwd(shape, q, k, v, lam, o, None, None, ws_f, stream)),
+                   ("bwd", lambda: la.la_bwd(shape, q, k, v, do, lam, dq, dk, dv, None, None, None, ws_b, stream,
+                                             fwd_workspace=ws_f))):
+        fn()
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        nrep = max(1, min(train_steps, 10))
+        s0.record(stream)
+        for _ in range(nrep):
+            fn()
+        s1.record(stream)
+        barrier()
+        split_ms[nm] = max_over_ranks(s0.elapsed_time(s1) / nrep)
+
     # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
     dw = inputs.WORKLOADS["decode"]
     gen = torch.Generator(dev)
@@ -339,7 +355,7 @@ def run_ours(args):
 
     # ---- the two smaller model shapes (reported beside the headline, same step and timing rules) ----
     others = {}
-    for name in ("385m", "1b"):
+    for name in ("pr1_ref", "385m", "1b"):
         ow = inputs.WORKLOADS[name]
         od_ = inputs.device_randn_like_workload(name, dev, seed=rank)
         oshape = la.make_shape(ow.B, ow.H, ow.N, ow.d, ow.e, ow.in_dtype, out_dtype)
@@ -372,12 +388,15 @@ def run_ours(args):
         oms = max_over_ranks(tot / osteps)
         oF = flops_per_token_head(ow.d)
         obytes = ow.token_heads * bytes_per_token_head(ow.d, ob, "step")
+        if ow.in_dtype == torch.float32:
+            obytes += ow.token_heads * 2 * 7 * ow.d  # q,k,v read twice and dO once, two bytes more each
         oroof = max(ow.token_heads * oF / (peaks["bf16_tflops_sustained"] * 1e12), obytes / (peaks["hbm_gbs"] * 1e9))
         others[name] = {"shape": "B=%d,H=%d,N=%d,d=e=%d" % (ow.B, ow.H, ow.N, ow.d), "ms_per_step": oms,
                         "tflops": world * ow.token_heads * oF / (oms * 1e-3) / 1e12,
                         "tokens_per_s": world * ow.B * ow.N / (oms * 1e-3),
                         "step_roofline_frac": oroof * 1e3 / oms, "l2": "flushed between timed steps",
-                        "kernels": "tcgen05 (one thread block per head and segment at d = 64, two at d = 128)"}
+                        "kernels": ("fp32 CUDA cores" if ow.in_dtype == torch.float32 else
+                                    "tcgen05 (one thread block per head and segment at d = 64, two at d = 128)")}
         del od_, oo, odq, odk, odv, owf, owb, flush
 
     clocks = sampler.stop() if rank == 0 else None
@@ -398,6 +417,7 @@ def run_ours(args):
             "tokens_per_s": world * w.B * w.N / (ms_step * 1e-3),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / args.steps for kname, (ms, _) in prof.items()},
+            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"),
             "roofline": {"kernel": "block walk (one launch each for O, dQ, dV, dK)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
