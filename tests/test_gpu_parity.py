@@ -477,3 +477,45 @@ def test_bounded_wait_expires_cleanly():
     assert_close(o, orc.fwd_rec(q, k, v, lam.double().numpy()), TOL_BF16, "o")
     with pytest.raises(la.LaError):
         la.selftest_bounded_wait(0)          # budget out of range: refused before any launch
+
+
+def test_decode_steps_replay_from_a_cuda_graph():
+    """la_decode_step keeps no host state between calls with the same arguments: a few steps captured into
+    a CUDA graph and replayed give bit-identical states and outputs to the same steps launched directly."""
+    B, H, d, steps = 2, 4, 128, 4
+    gen = torch.Generator("cpu")
+    gen.manual_seed(31)
+    qs = inputs.draw((steps, B, H, d), gen, "silu", torch.bfloat16).to(DEV)
+    ks = inputs.draw((steps, B, H, d), gen, "silu", torch.bfloat16).to(DEV)
+    vs = inputs.draw((steps, B, H, d), gen, "normal", torch.bfloat16).to(DEV)
+    lam = torch.tensor([1.0, 0.99, 0.7, 0.3])
+    kv0 = inputs.make_state(B, H, d, d, seed=32).to(DEV)
+    shape = la.make_shape(B, H, 1, d, d, torch.bfloat16, torch.float32)
+
+    kv_eager = kv0.clone()
+    o_eager = torch.empty((steps, B, H, d), dtype=torch.float32, device=DEV)
+    for s in range(steps):
+        la.la_decode_step(shape, qs[s], ks[s], vs[s], lam, kv_eager, o_eager[s])
+    torch.cuda.synchronize()
+
+    kv_graph = kv0.clone()
+    o_graph = torch.zeros_like(o_eager)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        la.la_decode_step(shape, qs[0], ks[0], vs[0], lam, kv_graph.clone(), o_graph[0].clone())  # warm-up outside capture
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            for s in range(steps):
+                la.la_decode_step(shape, qs[s], ks[s], vs[s], lam, kv_graph, o_graph[s])
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(kv_graph, kv_eager) and torch.equal(o_graph, o_eager)
+    # a second replay continues from the updated state, like four more direct steps
+    for s in range(steps):
+        la.la_decode_step(shape, qs[s], ks[s], vs[s], lam, kv_eager, o_eager[s])
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(kv_graph, kv_eager) and torch.equal(o_graph, o_eager)
