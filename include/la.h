@@ -19,10 +19,21 @@
  *     q,k,dq,dk [B,H,N,d]; v,o,dO,dv [B,H,N,e]; states [B,H,d,e] fp32 with
  *     kv[b,h,i,j] = sum_s lambda^(t-s) k_s[i] v_s[j].
  *   - Every tensor pointer is DEVICE memory, 16-byte aligned, owned by the caller.
- *     The library allocates no device memory, never frees, never synchronises
- *     the stream and keeps no mutable global state.  Inputs are not modified;
- *     outputs are fully overwritten; inputs and outputs must not alias (except
- *     the state of la_decode_step, which is updated in place).
+ *     The library allocates no device memory, never frees and never synchronises
+ *     the stream (la_device_status and la_profile_collect are the two calls that
+ *     wait, and say so).  Inputs are not modified; outputs are fully overwritten;
+ *     inputs and outputs must not alias (except the state of la_decode_step, which
+ *     is updated in place).
+ *   - State the library keeps between calls (everything else is per call): (1) one
+ *     failure flag per device, shared by all streams and callers, written by a
+ *     tensor-core block whose bounded wait expired and read by la_device_status;
+ *     (2) per device, the three side streams and events of la_fwd_bwd_host,
+ *     created on its first use; (3) the per-kernel timing records and the launch
+ *     counter of the benchmark helpers (process-wide, off by default);
+ *     (4) the fixed scratch array of la_fwd_noalloc, shared by all its callers on
+ *     a device.  la_fwd, la_bwd, la_bwd_reuse and la_decode_step touch none of
+ *     these except that their kernels may set (1), so concurrent calls from
+ *     several host threads on different streams are safe.
  *   - `lambda_host` is HOST memory: H floats, each finite and in (0, 1].  It is
  *     read during the call (validated, converted to -log2(lambda) in double) and
  *     passed to the kernels by value; it need not outlive the call.
@@ -57,7 +68,8 @@ typedef enum {
 typedef enum { LA_BF16 = 0, LA_F32 = 1 } la_dtype;
 
 /* Which kernels run.  AUTO picks the tensor-core kernels where they exist
- * (bf16 inputs, d = e = 128) and the fp32 CUDA-core kernels otherwise. */
+ * (bf16 inputs, d = e = 128 or d = e = 64) and the fp32 CUDA-core kernels otherwise
+ * (fp32 inputs).  TENSOR fails with LA_ERR_UNSUPPORTED where they do not exist. */
 typedef enum { LA_PATH_AUTO = 0, LA_PATH_SIMT = 1, LA_PATH_TENSOR = 2 } la_path;
 
 /* la_shape.precision, tensor-core path only: bf16 operands formed on chip from fp32
@@ -153,6 +165,10 @@ la_status la_decode_step(const la_shape* shape, const void* q, const void* k, co
  * device-wide synchronisation of an allocation, or a plug-in that is handed only tensor
  * pointers and a stream.  Inputs and outputs are still the caller's.
  *   - Every GPU that loads the library holds the 32 MiB array until the process exits.
+ *     With lazy module loading (the CUDA default) the array may only be materialised
+ *     when its address is first asked for, that is, inside the first call on a device:
+ *     make that warm-up call before the caller's own pool takes the rest of the
+ *     device memory, or it can fail with LA_ERR_CUDA for lack of room.
  *   - Shapes with la_workspace_bytes(LA_OP_FWD, shape) > LA_NOALLOC_SCRATCH_BYTES are
  *     rejected with LA_ERR_SCRATCH_LIMIT before anything is launched.
  *   - The first call on each device looks up the array's device address (once, with that
@@ -197,9 +213,14 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
  * Device-side failure flag (no counterpart in the paper).  The tensor-core kernels
  * never spin without limit: a thread block whose wait on a copy or on the tensor
  * cores expires records a code, drains what it started and returns, leaving its
- * part of the output unwritten.  This call copies the flag back (it blocks until
- * the device is idle), stores the raw code in *code if code is not NULL, clears
- * the flag, and returns LA_OK if no block failed, else LA_ERR_DEVICE_TIMEOUT.
+ * part of the output unwritten; la_fwd / la_bwd have returned LA_OK long before,
+ * so a caller that wants to know asks here.  The flag is one word per DEVICE, not
+ * per stream or per call: it keeps the first code any block recorded since it was
+ * last cleared, whoever launched that block.  This call waits until the whole
+ * device is idle (cudaDeviceSynchronize), takes the flag and clears it in one
+ * atomic exchange on the device, stores the raw code in *code if code is not
+ * NULL, and returns LA_OK if no block failed, else LA_ERR_DEVICE_TIMEOUT.  With
+ * several callers on one device, whoever calls first sees (and clears) the code.
  */
 la_status la_device_status(unsigned int* code);
 
@@ -229,9 +250,10 @@ unsigned long long la_launch_count(void);
  * CUDA events recorded on the caller's stream.  la_profile_collect waits for
  * those events, adds the elapsed milliseconds and launch counts per kernel kind
  * into ms[LA_NUM_KERNEL_KINDS] / launches[LA_NUM_KERNEL_KINDS] (both are
- * overwritten), releases the events and returns LA_OK.  This is the one piece of
- * mutable process-wide state in the library; it is off by default, guarded by a
- * mutex, and must not be enabled while a stream is being captured.
+ * overwritten), releases the events and returns LA_OK.  The records are
+ * process-wide state; profiling is off by default, guarded by a mutex, and must
+ * not be enabled while a stream is being captured.  It adds event records between
+ * the launches, so a loop timed as a whole should run with it off.
  */
 #define LA_KERNEL_PREPASS 0 /* segment-local states            */
 #define LA_KERNEL_SCAN 1    /* state scan across segments      */

@@ -24,7 +24,8 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
-           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse")
+           "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
+           "la_selftest_bounded_wait")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
 

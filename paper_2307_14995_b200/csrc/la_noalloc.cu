@@ -9,7 +9,10 @@
 // to ask.  For them the scratch lives here, in a fixed array in the library's own device image.
 //
 // Cost and limits: every GPU that loads the library holds LA_NOALLOC_SCRATCH_BYTES (32 MiB)
-// until the process exits.  A shape whose la_workspace_bytes(LA_OP_FWD, ..) exceeds that is
+// until the process exits.  With lazy module loading the array may only come into being when
+// its address is first asked for, so the first call on a device is the warm-up that can fail
+// for lack of room: make it before a pool takes the remaining device memory (and before any
+// stream capture).  A shape whose la_workspace_bytes(LA_OP_FWD, ..) exceeds that is
 // rejected with LA_ERR_SCRATCH_LIMIT before anything is launched.  All calls on a device share
 // the one array, so two calls that may overlap on the GPU (different streams) race on it; calls
 // on one stream are safe.  The array keeps whatever the previous call left, which is harmless:
@@ -42,7 +45,10 @@ la_status scratch_for_current_device(void** out) {
   std::lock_guard<std::mutex> lock(g_mu);
   if (!g_scratch_ptr[dev]) {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return LA_ERR_CUDA;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();  // leave no stale error behind in the runtime for the caller's next call
+      return LA_ERR_CUDA;
+    }
     g_scratch_ptr[dev] = p;
   }
   *out = g_scratch_ptr[dev];

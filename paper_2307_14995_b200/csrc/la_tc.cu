@@ -59,7 +59,8 @@
 
 namespace la {
 
-__device__ unsigned int g_tc_status = 0;  // first non-zero failure code of any block (0 = none)
+__device__ unsigned int g_tc_status = 0;       // first non-zero failure code of any block (0 = none)
+__device__ unsigned int g_tc_status_read = 0;  // where status_exchange_kernel leaves the value it took
 
 namespace {
 using namespace ptx;
@@ -170,30 +171,6 @@ __device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& lo
   lo = make_uint4(lw[0], lw[1], lw[2], lw[3]);
 }
 
-// Optional pipeline trace (debug builds with -DLA_TC_TRACE only): one chosen thread block stores
-// clock64() at named events, and every block of a walk launch its start/end time.
-#ifdef LA_TC_TRACE
-__device__ long long* g_tc_trace = nullptr;
-__device__ unsigned int g_tc_trace_block = 0;
-#define TC_TRACE(it, ev)                                                    \
-  do {                                                                      \
-    if (trace_ptr && (it) < 64) trace_ptr[(it) * 32 + (ev)] = clock64();    \
-  } while (0)
-__device__ unsigned long long* g_tc_cta_times = nullptr;  // [grid][2] start/end in ns (walk kernels only)
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define TC_CTA_TIME(slot)                                                                          \
-  do {                                                                                             \
-    if (!STATE_ONLY && g_tc_cta_times && threadIdx.x == 0) g_tc_cta_times[blockIdx.x * 2 + (slot)] = globaltimer_ns(); \
-  } while (0)
-#else
-#define TC_TRACE(it, ev) do { } while (0)
-#define TC_CTA_TIME(slot) do { } while (0)
-#endif
-
 #define TC_WAIT(barid, par, code)                                        \
   do {                                                                   \
     if (!wait_or_abort(&sm.bars[barid], (par), &sm.abort)) {             \
@@ -235,9 +212,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef LA_TC_TRACE
-  long long* const trace_ptr = (blockIdx.x == g_tc_trace_block) ? g_tc_trace : nullptr;
-#endif
   // D = 128: two thread blocks per (head, segment), one per half of the value columns.  D = 64: one
   // thread block; the feature halves 64..127 of the a and b tiles do not exist (the K steps over them are
   // skipped, and the second b panel, which M3 reads as rows 64..127 of b^T, is zeroed once below), so rows
@@ -290,7 +264,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_slot;
-  TC_CTA_TIME(0);
   bool issued_mma = false;
   uint32_t mma_elected = 0;  // set in the lane of warp 1 that issues the tensor-core instructions
   int armed_b[2] = {0, 0}, armed_c[2] = {0, 0};  // producer: uses armed per stage
@@ -329,12 +302,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           if (D == 128) tma_load_3d(&stg.a[1][0], &tm_a, &sm.bars[FULL_B0 + s], 64, t0, bh);
         }
         armed_b[s] = (it >> 1) + 1;
-        TC_TRACE(it, 0);
         if (it >= 2) TC_WAIT(C_FREE0 + s, prev, 2);
         mbar_arrive_expect_tx(&sm.bars[FULL_C0 + s], 16384);
         tma_load_3d(&stg.c[0], &tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, bh);
         armed_c[s] = (it >> 1) + 1;
-        TC_TRACE(it, 1);
       }
     }
   } else if (warp == 1 && STATE_ONLY) {
@@ -403,11 +374,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           const uint32_t c0 = smem_u32(&sm.st[s].c[0]);
           const uint32_t col_p = s ? COL_S1 : COL_S0;
           // M3: dZ = b^T [fc_hi | fc_lo]  (needs the previous dZ to have been read)
-          TC_TRACE(it, 15);
           // Z_READY: the state operand of this block AND fc of this block are in place (the Z group forms fc first)
           TC_WAIT(Z_READY, par1, 12);
           tc_fence_after_sync();
-          TC_TRACE(it, 3);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
             umma_bf16(tmem + COL_DZ, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
@@ -419,12 +388,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                         umma_desc_sw128(fh0 + 16384 + k * 2048, 16384, 1024), ID_MN64, 1);
           }
           umma_commit(&sm.bars[DZ_READY]);
-          TC_TRACE(it, 16);
           // M2: O_inter = a Z   (state after the previous block / the entry state)
           // this O_inter buffer was last read for block it-2; that read was already awaited before M4(it-1)
           const uint32_t col_oe = (it & 1) ? COL_OE1 : COL_OE0;
           tc_fence_after_sync();
-          TC_TRACE(it, 5);
 #pragma unroll
           for (int k = 0; k < KD; ++k) {
             const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
@@ -440,7 +407,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             }
           }
           umma_commit(&sm.bars[A_FREE0 + s]);  // M1 and M2 of this block are done with the a tile
-          TC_TRACE(it, 19);
           // M1 of the next block, into the other S/P buffer
           if (it + 1 < nblk) {
             const int s1 = s ^ 1;
@@ -448,7 +414,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             const uint32_t an = smem_u32(&sm.st[s1].a[0][0]), bn = smem_u32(&sm.st[s1].b[0][0]);
             TC_WAIT(FULL_B0 + s1, parn, 11);  // a and b of the next block
             tc_fence_after_sync();
-            TC_TRACE(it, 4);
 #pragma unroll
             for (int k = 0; k < KD; ++k) {
               const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
@@ -458,11 +423,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
             umma_commit(&sm.bars[S_READY0 + s1]);
           }
           // M4: O_intra = P c, P read from tensor memory (K step k: hi pairs at column 16k, lo pairs at 16k+8)
-          TC_TRACE(it, 20);
           TC_WAIT(P_READY0 + s, par2, 14);  // P is written and the accumulators of the previous block have been read
           TC_WAIT(FULL_C0 + s, par2, 15);
           tc_fence_after_sync();
-          TC_TRACE(it, 6);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
             umma_bf16_ts(tmem + COL_OI, tmem + col_p + 16 * k, umma_desc_sw128(c0 + k * 2048, 16384, 1024), ID_KN,
@@ -474,7 +437,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
                            ID_KN, 1);
           }
           umma_commit(&sm.bars[O_READY]);
-          TC_TRACE(it, 21);
         }
       }
     }
@@ -556,7 +518,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         const uint32_t colS = lane_addr + (s ? COL_S1 : COL_S0);
         TC_WAIT_WARP(S_READY0 + s, (it >> 1) & 1, 17);
         tc_fence_after_sync();
-        if (tid == 224) TC_TRACE(it, 7);
 #pragma unroll 1
         for (int ci = 0; ci < 2; ++ci) {
           const int cc = half * 2 + ci;
@@ -593,7 +554,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         tmem_st_wait();
         tc_fence_before_sync();
         WARP_ARRIVE(P_READY0 + s);
-        if (tid == 224) TC_TRACE(it, 8);
       }
     }
   } else if (warp >= 12 && warp < 20) {
@@ -690,7 +650,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         // ---- Z <- Gamma Z + dZ ----
         TC_WAIT_WARP(DZ_READY, it & 1, 22);
         tc_fence_after_sync();
-        if (tid == 384) TC_TRACE(it, 9);
         {
           const float gamma = exp2f(-s2 * (float)Cr);
 #pragma unroll
@@ -707,12 +666,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           // DZ_READY also says M3 of this block is done, so the fc buffer may be rewritten
           make_fc(cnext, state_factor(it + 1), sm.fc_hi, sm.fc_lo);
           if (it + 2 < nblk) c_from_global(it + 2, cnext);
-          if (tid == 384) TC_TRACE(it, 10);
           // A_FREE of this block's stage: M2 of this block is done, so it has read the old state operand
           TC_WAIT_WARP(A_FREE0 + (it & 1), (it >> 1) & 1, 23);
           write_state_operand();
           WARP_ARRIVE(Z_READY);
-          if (tid == 384) TC_TRACE(it, 11);
         }
       }
       const bool last_processed = REV ? (seg == 0) : (seg == args.nseg - 1);
@@ -743,7 +700,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         // O_READY: every MMA up to M4 of this block is done
         TC_WAIT_WARP(O_READY, it & 1, 25);
         tc_fence_after_sync();
-        if (tid == 736) TC_TRACE(it, 12);
         constexpr int PASSES = (sizeof(TOut) == 4) ? 2 : 1;  // 128 bytes of each output row per pass
         constexpr int PIECES = (sizeof(TOut) == 4) ? 2 : 4;  // 16-column accumulator pieces per pass
 #pragma unroll
@@ -760,7 +716,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
               tc_fence_before_sync();
               // both accumulators are in registers now: M4 of the next block may overwrite O_intra
               if (it + 1 < nblk) WARP_ARRIVE(P_READY0 + (s ^ 1));
-              if (tid == 736) TC_TRACE(it, 13);
             }
             if (sizeof(TOut) == 4) {
 #pragma unroll
@@ -802,7 +757,6 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           tma_store_wait_read();
           mbar_arrive(&sm.bars[C_FREE0 + s]);  // the c tile of this stage may be reloaded
         }
-        if (tid == 736) TC_TRACE(it, 14);
       }
     }
   }
@@ -826,7 +780,6 @@ teardown:
   }
   tc_fence_before_sync();
   __syncthreads();
-  TC_CTA_TIME(1);
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
@@ -930,29 +883,24 @@ cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, 
   return D == 128 ? launch_prepass_d<128>(args, tab, precision, stream) : launch_prepass_d<64>(args, tab, precision, stream);
 }
 
-#ifdef LA_TC_TRACE
-extern "C" void la_debug_set_trace(long long* device_buffer, unsigned int block) {
-  cudaMemcpyToSymbol(g_tc_trace, &device_buffer, sizeof(device_buffer));
-  cudaMemcpyToSymbol(g_tc_trace_block, &block, sizeof(block));
-}
-extern "C" void la_debug_set_cta_times(unsigned long long* device_buffer) {
-  cudaMemcpyToSymbol(g_tc_cta_times, &device_buffer, sizeof(device_buffer));
-}
-#endif
-
 cudaError_t launch_bounded_wait_selftest(long long budget_clocks, cudaStream_t stream) {
   bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(budget_clocks);
   count_launch();
   return cudaGetLastError();
 }
 
+// Reads the failure flag and clears it in one atomic exchange on the device, so that a code recorded between
+// a separate read and a separate clear cannot be lost.
+__global__ void status_exchange_kernel(bool clear) {
+  g_tc_status_read = clear ? atomicExch(&g_tc_status, 0u) : atomicAdd(&g_tc_status, 0u);
+}
+
 unsigned int tc_read_status(bool clear) {
   unsigned int v = 0;
-  if (cudaMemcpyFromSymbol(&v, g_tc_status, sizeof(v)) != cudaSuccess) return 0xFFFFFFFFu;
-  if (clear && v != 0) {
-    const unsigned int zero = 0;
-    cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(zero));
-  }
+  status_exchange_kernel<<<1, 1, 0, cudaStreamPerThread>>>(clear);
+  if (cudaGetLastError() != cudaSuccess) return 0xFFFFFFFFu;
+  if (cudaStreamSynchronize(cudaStreamPerThread) != cudaSuccess) return 0xFFFFFFFFu;
+  if (cudaMemcpyFromSymbol(&v, g_tc_status_read, sizeof(v)) != cudaSuccess) return 0xFFFFFFFFu;
   return v;
 }
 

@@ -37,8 +37,10 @@ def test_exports_every_declared_symbol(lib):
 
 def test_version_and_status_strings(lib):
     assert la.version() >= 100
-    seen = {la.status_string(c) for c in range(7)}
-    assert len(seen) == 7 and "ok" in seen
+    seen = {la.status_string(c) for c in range(8)}
+    assert len(seen) == 8 and "ok" in seen and "unknown status" not in seen
+    assert "scratch" in la.status_string(7)          # LA_ERR_SCRATCH_LIMIT
+    assert la.status_string(8) == "unknown status"
 
 
 def shape(**kw):

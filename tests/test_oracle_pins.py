@@ -124,6 +124,42 @@ def test_no_decay_is_prefix_sum():
     for got in (orc.bwd_rec(q, k, v, do, lam), orc.bwd_quad(q, k, v, do, lam)):
         for g, w in zip(got, want_g):
             assert relerr(g, w) < 1e-14
+    # the state handed out is the last prefix sum, rows = key feature, columns = value feature
+    # (d = 4 and e = 5 differ, so a transposed convention cannot pass)
+    _, kv_out = orc.fwd_rec(q, k, v, lam, want_state=True)
+    assert kv_out.shape == (1, 2, 4, 5)
+    assert relerr(kv_out, kv_prefix[:, :, -1]) < 1e-14
+
+
+@pytest.mark.parametrize("lam_val", [0.9, 0.35])
+def test_state_orientation_and_decay_by_explicit_sum(lam_val):
+    """kv_out[i, j] = sum_s lambda^(N-1-s) k_s[i] v_s[j], written as a plain numpy loop over s; with a
+    state handed in, it enters as lambda^N kv_in, and grad_kv_in = lambda^N grad_kv_out +
+    sum_t lambda^(t+1) q_t do_t^T in the same orientation (d != e throughout)."""
+    B, H, N, d, e = 1, 2, 21, 3, 5
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=51)
+    lam = np.array([lam_val, 1.0])
+    qn, kn, vn, don = (x.double().numpy() for x in (q, k, v, do))
+    rng = np.random.default_rng(3)
+    kv_in = rng.standard_normal((B, H, d, e))
+    gko = rng.standard_normal((B, H, d, e))
+    want_kv = np.zeros((B, H, d, e))
+    want_gin = np.zeros((B, H, d, e))
+    for h in range(H):
+        for s in range(N):
+            want_kv[0, h] += lam[h] ** (N - 1 - s) * np.outer(kn[0, h, s], vn[0, h, s])
+            want_gin[0, h] += lam[h] ** (s + 1) * np.outer(qn[0, h, s], don[0, h, s])
+    _, kv0 = orc.fwd_rec(q, k, v, lam, want_state=True)
+    assert relerr(kv0, want_kv) < 1e-14
+    decay_n = (lam ** N)[None, :, None, None]
+    o1, kv1 = orc.fwd_rec(q, k, v, lam, kv_in=kv_in, want_state=True)
+    assert relerr(kv1, want_kv + decay_n * kv_in) < 1e-14
+    # o_t with a state handed in gains lambda^(t+1) kv_in^T q_t
+    t = np.arange(N)
+    extra = np.einsum("bhti,bhij->bhtj", qn, kv_in) * (lam[None, :, None] ** (t[None, None, :] + 1))[..., None]
+    assert relerr(o1 - orc.fwd_rec(q, k, v, lam), extra) < 1e-13
+    *_, gin = orc.bwd_rec(q, k, v, do, lam, kv_in=kv_in, grad_kv_out=gko, want_state_grad=True)
+    assert relerr(gin, want_gin + decay_n * gko) < 1e-14
 
 
 def test_fast_decay_limit_is_diagonal():
@@ -243,6 +279,32 @@ def test_linearity_scaling():
     lam = np.array([0.75])
     base = orc.fwd_rec(q, k, v, lam)
     assert relerr(orc.fwd_rec(2 * q, 4 * k, 0.5 * v, lam), 4 * base) < 1e-15
+
+
+# --- random tiny shapes: both forms of the oracle against the literal loops -----------
+from hypothesis import given, settings, strategies as st  # noqa: E402
+
+
+@settings(max_examples=25, deadline=None)
+@given(N=st.integers(1, 9), d=st.integers(1, 4), e=st.integers(1, 4), H=st.integers(1, 2),
+       lam0=st.sampled_from([1.0, 0.97, 0.5, 0.05, 1e-30]), seed=st.integers(0, 10_000))
+def test_random_tiny_shapes_against_brute_force(N, d, e, H, lam0, seed):
+    """Any N >= 1 and d != e: recurrence == quadratic form == literal loops (forward), and the two
+    backward forms agree with each other and satisfy the Euler identities."""
+    q, k, v, do = rand_inputs(1, H, N, d, e, seed=seed)
+    lam = np.array([lam0, 0.8][:H])
+    want = brute_forward(q.numpy(), k.numpy(), v.numpy(), lam)
+    o_rec, o_quad = orc.fwd_rec(q, k, v, lam), orc.fwd_quad(q, k, v, lam)
+    scale = np.sqrt(np.mean(want * want)) + 1e-30
+    assert np.max(np.abs(o_rec - want)) <= 1e-13 * scale + 1e-300
+    assert np.max(np.abs(o_quad - want)) <= 1e-13 * scale + 1e-300
+    g_rec, g_quad = orc.bwd_rec(q, k, v, do, lam), orc.bwd_quad(q, k, v, do, lam)
+    for a, b in zip(g_rec, g_quad):
+        assert np.max(np.abs(a - b)) <= 1e-12 * (np.sqrt(np.mean(b * b)) + 1e-30) + 1e-300
+    qn, kn, vn, don = (x.double().numpy() for x in (q, k, v, do))
+    ref = np.sum(want * don, axis=(2, 3))
+    for a, b in ((qn, g_rec[0]), (kn, g_rec[1]), (vn, g_rec[2])):
+        assert np.allclose(np.sum(a * b, axis=(2, 3)), ref, rtol=1e-10, atol=1e-12 * (np.abs(ref).max() + 1e-30))
 
 
 # --- state hand-over, decode, causality ---------------------------------------------

@@ -2,8 +2,8 @@
 (all memory already given to their own pool, no allocator at hand, or no tolerance for the
 device-wide synchronisation an allocation brings).  Its scratch is a fixed array inside the
 library, so this file checks, through the C ABI, that it gives what la_fwd gives with a
-caller-allocated workspace -- twice in a row, because the second call finds the first call's
-leftovers in the shared scratch.  Collected last on purpose (file name), and self-contained so
+caller-allocated workspace -- and what the CPU oracle's token recurrence gives -- twice in a row,
+because the second call finds the first call's leftovers in the shared scratch.  Collected last on purpose (file name), and self-contained so
 that it passes alone in a fresh process as well as after the rest of the suite."""
 import ctypes
 
@@ -11,6 +11,7 @@ import pytest
 import torch
 
 from la_check import TOL_BF16, assert_close
+from oracle import la_oracle as orc
 from paper_2307_14995_b200 import binding as la, inputs
 
 
@@ -43,6 +44,8 @@ def test_noalloc_matches_la_fwd_twice_in_a_row(d, path):
     kv_ref = torch.empty((B, H, d, d), dtype=torch.float32, device=dev)
     la.la_fwd(shape, qg, kg, vg, lam, o_ref, kv_in, kv_ref, la.alloc_workspace(la.LA_OP_FWD, shape, dev))
     torch.cuda.synchronize()
+    o_orc, kv_orc = orc.fwd_rec(q, k, v, lam.double().numpy(), kv_in=kv_in.double().cpu().numpy(), want_state=True)
+    tol = TOL_BF16 if path != la.LA_PATH_SIMT else 1e-4
 
     for attempt in range(2):
         o = torch.full((B, H, N, d), float("nan"), dtype=torch.float32, device=dev)
@@ -59,3 +62,5 @@ def test_noalloc_matches_la_fwd_twice_in_a_row(d, path):
         assert_close(o, o_ref.double().cpu().numpy(), TOL_BF16, "o, call %d" % attempt)
         assert_close(kv, kv_ref.double().cpu().numpy(), TOL_BF16, "kv_out, call %d" % attempt)
         assert torch.equal(o, o_ref) and torch.equal(kv, kv_ref)  # same kernels, same order: bitwise equal
+        assert_close(o, o_orc, tol, "o vs oracle, call %d" % attempt)
+        assert_close(kv, kv_orc, tol, "kv_out vs oracle, call %d" % attempt)
