@@ -259,7 +259,8 @@ unsigned long long la_launch_count(void);
 #define LA_KERNEL_SCAN 1    /* state scan across segments      */
 #define LA_KERNEL_WALK 2    /* block walk producing o/dq/dk/dv */
 #define LA_KERNEL_DECODE 3  /* recurrent decode step           */
-#define LA_NUM_KERNEL_KINDS 4
+#define LA_KERNEL_WALK_PAIR 4 /* the dV and dK walks of the backward pass in one launch */
+#define LA_NUM_KERNEL_KINDS 5
 void la_profile_enable(int on);
 la_status la_profile_collect(double* ms, unsigned long long* launches);
 

@@ -27,7 +27,7 @@ EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_de
            "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
            "la_selftest_bounded_wait")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
-KERNEL_KINDS = ("prepass", "scan", "walk", "decode")
+KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair")
 
 
 class LaShape(ctypes.Structure):

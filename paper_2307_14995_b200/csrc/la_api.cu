@@ -185,9 +185,8 @@ cudaError_t run_scan(const la_shape* s, const Plan& p, const DecayTable& tab, fl
   return launch_scan(sa, tab, st);
 }
 
-cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, const void* a,
-                     const void* b, const void* c, void* out, const float* entry, float* final_out,
-                     int reverse, cudaStream_t st) {
+OpArgs walk_args(const la_shape* s, const Plan& p, const void* a, const void* b, const void* c, void* out,
+                 const float* entry, float* final_out, int reverse) {
   OpArgs args{};
   args.a = a;
   args.b = b;
@@ -201,6 +200,13 @@ cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, co
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
+  return args;
+}
+
+cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, const void* a,
+                     const void* b, const void* c, void* out, const float* entry, float* final_out,
+                     int reverse, cudaStream_t st) {
+  const OpArgs args = walk_args(s, p, a, b, c, out, entry, final_out, reverse);
   if (p.tensor) return launch_tc_walk(args, tab, s->d, (int)s->out_dtype, p.precision, st);
   return launch_simt_walk(args, tab, s->d, s->e, (int)s->in_dtype, (int)s->out_dtype, st);
 }
@@ -318,8 +324,17 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
     entry_v = buf_e;
     entry_k = buf_et;
   }
-  LA_TRY_CUDA(run_walk(shape, p, tab, k, q, d_o, dv, entry_v, grad_kv_in, 1, cs));
-  LA_TRY_CUDA(run_walk(shape, p, tab, v, d_o, q, dk, entry_k, nullptr, 1, cs));
+  if (p.tensor && tc_pair_enabled()) {
+    // both reverse walks in one launch: together they read Q, K, V and dO, and the thread blocks of the two are
+    // interleaved so that each of those tiles comes from HBM once (Algorithm 4 accumulates dK_j and dV_j in the
+    // same outer iteration for the same reason)
+    const OpArgs walk_v = walk_args(shape, p, k, q, d_o, dv, entry_v, grad_kv_in, 1);
+    const OpArgs walk_k = walk_args(shape, p, v, d_o, q, dk, entry_k, nullptr, 1);
+    LA_TRY_CUDA(launch_tc_walk_pair(walk_v, walk_k, tab, shape->d, (int)shape->out_dtype, p.precision, cs));
+  } else {
+    LA_TRY_CUDA(run_walk(shape, p, tab, k, q, d_o, dv, entry_v, grad_kv_in, 1, cs));
+    LA_TRY_CUDA(run_walk(shape, p, tab, v, d_o, q, dk, entry_k, nullptr, 1, cs));
+  }
   return LA_OK;
 }
 

@@ -77,6 +77,11 @@ cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv
 bool tc_supported();
 cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int out_dt, int precision,
                            cudaStream_t stream);
+// Two walks of the same direction over the same tokens (same N, BH, segments) in one launch; the thread blocks of
+// the two are interleaved so that tiles both read come from HBM once.
+bool tc_pair_enabled();
+cudaError_t launch_tc_walk_pair(const OpArgs& first, const OpArgs& second, const DecayTable& tab, int D, int out_dt,
+                                int precision, cudaStream_t stream);
 cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, int precision,
                               cudaStream_t stream);
 
@@ -99,7 +104,7 @@ struct KernelTimer {
   cudaEvent_t start_;
   bool active_;
 };
-enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_NUM = 4 };
+enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_WALK_PAIR = 4, K_NUM = 5 };
 
 // ---- small device helpers --------------------------------------------------
 __device__ __forceinline__ float decay_pow(float s2, float n) {

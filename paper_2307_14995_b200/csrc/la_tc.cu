@@ -54,6 +54,8 @@
 // K-major in M1 and MN-major (as b^T) in M3 from the same bytes.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "la_common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -97,14 +99,26 @@ struct alignas(1024) TcSmem {
   int abort;
 };
 
-struct TcArgs {
+// One launch carries one job, or two jobs that walk the same tokens in the same direction (the dV and dK walks of
+// the backward pass: they read the same four tensors, so the second read of each tile is an L2 hit).
+struct TcJob {
   const void* c;  // value-like tensor, also read row-wise straight from global memory by the Z group
   void* out;
   const float* entry;
-  float* local_out;
   float* final_out;
+};
+
+struct TcMaps {
+  CUtensorMap a, b, c, out;
+};
+
+struct TcArgs {
+  TcJob job[2];
+  float* local_out;
+  int njobs;
   int BH, H, N, seg_len, nseg;
   int precision;
+  int tune;  // experiment switches (environment variable LA_TC_TUNE, read once)
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
@@ -201,10 +215,9 @@ __device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& lo
     if (lane == 0) mbar_arrive(&sm.bars[barid]);         \
   } while (0)
 
-template <bool REV, bool STATE_ONLY, typename TOut, int D>
+template <bool REV, bool STATE_ONLY, typename TOut, int D, int NJOBS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-          const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_out, const TcArgs args,
+tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps maps1, const TcArgs args,
           const DecayTable tab) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler keeps
@@ -218,13 +231,43 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
   // 64..127 of the state stay zero and are neither loaded nor stored.
   static_assert(D == 64 || D == 128, "feature dimension");
   constexpr int KD = D / 16;  // K steps over the feature dimension
-  const int ehalf = (D == 128) ? (int)(blockIdx.x & 1) : 0;
-  const int segid = (D == 128) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  // With two jobs the thread blocks of one (head, segment) -- both jobs, both value halves -- have adjacent
+  // indices, so they run at the same time and share their tiles through L2.
+  const int jobid = (NJOBS == 2) ? (int)(blockIdx.x & 1) : 0;
+  const unsigned bidx = (NJOBS == 2) ? (blockIdx.x >> 1) : blockIdx.x;
+  TcJob job = args.job[0];
+  if (NJOBS == 2 && jobid) job = args.job[1];
+  const CUtensorMap* const tm_a = (NJOBS == 2 && jobid) ? &maps1.a : &maps0.a;
+  const CUtensorMap* const tm_b = (NJOBS == 2 && jobid) ? &maps1.b : &maps0.b;
+  const CUtensorMap* const tm_c = (NJOBS == 2 && jobid) ? &maps1.c : &maps0.c;
+  const CUtensorMap* const tm_out = (NJOBS == 2 && jobid) ? &maps1.out : &maps0.out;
+  const int ehalf = (D == 128) ? (int)(bidx & 1) : 0;
+  const int segid = (D == 128) ? (int)(bidx >> 1) : (int)bidx;
   const int bh = segid / args.nseg, seg = segid % args.nseg;
   const int seg_t0 = seg * args.seg_len;
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
-  const int nblk = (seg_t1 - seg_t0 + 127) >> 7;
   const float s2 = (float)tab.s2[bh % args.H];
+  int nblk = (seg_t1 - seg_t0 + 127) >> 7;
+  int it0 = 0;  // forward pre-pass: index of the first block that is walked
+  if (STATE_ONLY && s2 > 0.f) {
+    // The pre-pass weighs every token by its decay to the edge the state leaves the segment through.  Once
+    // s2 * distance exceeds 150 that weight is exactly zero in fp32 (exp2f underflows past the smallest
+    // subnormal), so whole blocks far from the edge add exactly nothing and are not loaded at all: the blocks
+    // kept are those whose nearest token is within 160 / s2 + 128 tokens of the edge (the margin makes the
+    // skipped weights zero whatever the rounding of this bound).  Results are those of walking every block.
+    const float reach = 160.f / s2;  // tokens
+    int keep;
+    if (REV) {
+      keep = (int)fminf(ceilf((reach - 1.f) * (1.f / 128.f)) + 2.f, (float)nblk);
+    } else {
+      const float x = ((float)(seg_t1 - seg_t0) - reach) * (1.f / 128.f);  // blocks before the reach
+      const int skip = max(0, min(nblk - 1, (int)floorf(x - 1.f)));
+      keep = nblk - skip;
+      it0 = skip;
+    }
+    keep = max(1, min(keep, nblk));
+    nblk = keep;  // the reverse pre-pass walks blocks nblk-1 .. 0, the forward one it0 .. it0+nblk-1
+  }
   const bool split_p = (args.precision & 1) != 0;
   const bool split_z = (args.precision & 2) != 0;
   // lambda == 1: the decayed rows equal the bf16 inputs, their lo term is identically zero
@@ -246,10 +289,10 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     }
     sm.abort = 0;
     fence_mbar_init();
-    tma_prefetch_desc(&tm_a);
-    tma_prefetch_desc(&tm_b);
-    tma_prefetch_desc(&tm_c);
-    if (!STATE_ONLY) tma_prefetch_desc(&tm_out);
+    tma_prefetch_desc(tm_a);
+    tma_prefetch_desc(tm_b);
+    tma_prefetch_desc(tm_c);
+    if (!STATE_ONLY) tma_prefetch_desc(tm_out);
   }
   if (warp == 1) {
     tmem_alloc(&sm.tmem_slot, TMEM_COLS);
@@ -274,37 +317,37 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       for (int it = 0; it < nblk; ++it) {
         const int s = it & 1;
         const uint32_t prev = ((it >> 1) - 1) & 1;  // parity of this stage's previous use
-        const int blk = REV ? (nblk - 1 - it) : it;
+        const int blk = REV ? (nblk - 1 - it) : (it + it0);
         const int t0 = seg_t0 + blk * 128;
         Stage& stg = sm.st[s];
         // State-only kernel: its two stages hold less than what must be in flight to cover the latency of
         // HBM, so the tiles two blocks ahead are pulled into L2 now and the loads proper become L2 hits
         // (measured: 0.276 -> 0.245 ms per launch; the same in the walk kernel made it slower).
         if (STATE_ONLY && it + 2 < nblk) {
-          const int tp = seg_t0 + (REV ? (nblk - 3 - it) : (it + 2)) * 128;
-          tma_prefetch_3d(&tm_b, 0, tp, bh);
-          if (D == 128) tma_prefetch_3d(&tm_b, 64, tp, bh);
-          tma_prefetch_3d(&tm_c, ehalf * 64, tp, bh);
+          const int tp = seg_t0 + (REV ? (nblk - 3 - it) : (it + 2 + it0)) * 128;
+          tma_prefetch_3d(tm_b, 0, tp, bh);
+          if (D == 128) tma_prefetch_3d(tm_b, 64, tp, bh);
+          tma_prefetch_3d(tm_c, ehalf * 64, tp, bh);
         }
         if (STATE_ONLY) {
           if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
           mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 256);
-          tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+          tma_load_3d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
+          if (D == 128) tma_load_3d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
         } else {
           // walk kernel: the a and b tiles of a stage travel together (one barrier for both, FULL_B); A_FREE
           // is committed after M2, the last product of the block that reads either of them
           if (it >= 2) TC_WAIT(A_FREE0 + s, prev, 3);
           mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 512);
-          tma_load_3d(&stg.b[0][0], &tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.b[1][0], &tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
-          tma_load_3d(&stg.a[0][0], &tm_a, &sm.bars[FULL_B0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.a[1][0], &tm_a, &sm.bars[FULL_B0 + s], 64, t0, bh);
+          tma_load_3d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
+          if (D == 128) tma_load_3d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+          tma_load_3d(&stg.a[0][0], tm_a, &sm.bars[FULL_B0 + s], 0, t0, bh);
+          if (D == 128) tma_load_3d(&stg.a[1][0], tm_a, &sm.bars[FULL_B0 + s], 64, t0, bh);
         }
         armed_b[s] = (it >> 1) + 1;
         if (it >= 2) TC_WAIT(C_FREE0 + s, prev, 2);
         mbar_arrive_expect_tx(&sm.bars[FULL_C0 + s], 16384);
-        tma_load_3d(&stg.c[0], &tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, bh);
+        tma_load_3d(&stg.c[0], tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, bh);
         armed_c[s] = (it >> 1) + 1;
       }
     }
@@ -342,6 +385,60 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         umma_commit_if(&sm.bars[FC_FREE0 + s], go);
       }
       umma_commit_if(&sm.bars[DZ_READY], go);
+    }
+  } else if (warp == 1 && (args.tune & 4)) {
+    // ------------------------------------ MMA issuer, walk kernel, warp-convergent form ------------------------------------
+    // The same schedule as the single-lane form below, run by all 32 lanes together; only the tensor-core
+    // instructions and their commits are predicated on one elected lane.
+    {
+      constexpr uint32_t ID_S = umma_idesc_bf16(128, 128, false, false);
+      constexpr uint32_t ID_KN = umma_idesc_bf16(128, 64, false, true);
+      constexpr uint32_t ID_MN64 = umma_idesc_bf16(128, 64, true, true);
+      constexpr uint32_t HI = UMMA_DESC_HI_SBO1024;
+      const uint32_t go = elect_one();
+      mma_elected = go;
+      // low descriptor halves.  K-major tiles (a, b in M1; a in M2): K step k adds (k >> 2) * 16 KB + (k & 3) * 32 B;
+      // MN-major tiles (b^T in M3, fc, the state operand, c): K step k adds k * 2 KB.
+      const uint32_t ak0 = umma_desc_lo(smem_u32(&sm.st[0].a[0][0]), 16), ak1 = umma_desc_lo(smem_u32(&sm.st[1].a[0][0]), 16);
+      const uint32_t bk0 = umma_desc_lo(smem_u32(&sm.st[0].b[0][0]), 16), bk1 = umma_desc_lo(smem_u32(&sm.st[1].b[0][0]), 16);
+      const uint32_t bm0 = umma_desc_lo(smem_u32(&sm.st[0].b[0][0]), 16384), bm1 = umma_desc_lo(smem_u32(&sm.st[1].b[0][0]), 16384);
+      const uint32_t cm0 = umma_desc_lo(smem_u32(&sm.st[0].c[0]), 16384), cm1 = umma_desc_lo(smem_u32(&sm.st[1].c[0]), 16384);
+      const uint32_t fh = umma_desc_lo(smem_u32(&sm.fc_hi[0]), 16384), fl = umma_desc_lo(smem_u32(&sm.fc_lo[0]), 16384);
+      const uint32_t zh = umma_desc_lo(smem_u32(&sm.z_hi[0]), 16384), zl = umma_desc_lo(smem_u32(&sm.z_lo[0]), 16384);
+      TC_WAIT_WARP(FULL_B0, 0, 7);
+      tc_fence_after_sync();
+      umma_group_ss<KD, true, true>(tmem + COL_S0, ak0, bk0, HI, ID_S, 0, go);
+      issued_mma = true;
+      umma_commit_if(&sm.bars[S_READY0], go);
+      for (int it = 0; it < nblk; ++it) {
+        const int s = it & 1;
+        const uint32_t par1 = it & 1, par2 = (it >> 1) & 1;
+        const uint32_t col_p = s ? COL_S1 : COL_S0;
+        const uint32_t aks = s ? ak1 : ak0, bms = s ? bm1 : bm0, cms = s ? cm1 : cm0;
+        const uint32_t akn = s ? ak0 : ak1, bkn = s ? bk0 : bk1;  // the other stage (next block)
+        TC_WAIT_WARP(Z_READY, par1, 12);
+        tc_fence_after_sync();
+        umma_group_ss<8, false, false>(tmem + COL_DZ, bms, fh, HI, ID_MN64, 0, go);
+        if (split_c) umma_group_ss<8, false, false>(tmem + COL_DZ, bms, fl, HI, ID_MN64, 1, go);
+        umma_commit_if(&sm.bars[DZ_READY], go);
+        const uint32_t col_oe = (it & 1) ? COL_OE1 : COL_OE0;
+        umma_group_ss<KD, true, false>(tmem + col_oe, aks, zh, HI, ID_KN, 0, go);
+        if (split_z) umma_group_ss<KD, true, false>(tmem + col_oe, aks, zl, HI, ID_KN, 1, go);
+        umma_commit_if(&sm.bars[A_FREE0 + s], go);
+        if (it + 1 < nblk) {
+          const int s1 = s ^ 1;
+          TC_WAIT_WARP(FULL_B0 + s1, ((it + 1) >> 1) & 1, 11);
+          tc_fence_after_sync();
+          umma_group_ss<KD, true, true>(tmem + (s1 ? COL_S1 : COL_S0), akn, bkn, HI, ID_S, 0, go);
+          umma_commit_if(&sm.bars[S_READY0 + s1], go);
+        }
+        TC_WAIT_WARP(P_READY0 + s, par2, 14);
+        TC_WAIT_WARP(FULL_C0 + s, par2, 15);
+        tc_fence_after_sync();
+        umma_group_ts8(tmem + COL_OI, tmem + col_p, cms, HI, ID_KN, 0, go);
+        if (split_p) umma_group_ts8(tmem + COL_OI, tmem + col_p + 8, cms, HI, ID_KN, 1, go);
+        umma_commit_if(&sm.bars[O_READY], go);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------ MMA issuer, walk kernel ------------------------------------
@@ -448,7 +545,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
     const int r = q * 32 + lane;
     for (int it = 0; it < nblk; ++it) {
       const int s = it & 1;
-      const int blk = REV ? (nblk - 1 - it) : it;
+      const int blk = REV ? (nblk - 1 - it) : (it + it0);
       const int t0 = seg_t0 + blk * 128;
       // decay from token t0 + r to the edge of the segment that the state leaves through
       float f = 0.f;
@@ -598,7 +695,7 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
       const int blk = REV ? (nblk - 1 - it) : it;
       const int t = seg_t0 + blk * 128 + r;
       if (t < args.N) {
-        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(args.c) +
+        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
                                                           ((size_t)bh * args.N + t) * D + ehalf * 64 + zh * 32);
 #pragma unroll
         for (int x = 0; x < 4; ++x) raw[x] = __ldg(src + x);
@@ -610,9 +707,9 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
 
     {
       float zreg[32];
-      if (args.entry && r < D) {
+      if (job.entry && r < D) {
         const float4* src = reinterpret_cast<const float4*>(
-            args.entry + ((size_t)bh * args.nseg + seg) * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32);
+            job.entry + ((size_t)bh * args.nseg + seg) * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32);
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
           const float4 v = __ldg(src + x);
@@ -673,8 +770,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         }
       }
       const bool last_processed = REV ? (seg == 0) : (seg == args.nseg - 1);
-      if (args.final_out && last_processed && r < D) {
-        float* dst = args.final_out + (size_t)bh * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32;
+      if (job.final_out && last_processed && r < D) {
+        float* dst = job.final_out + (size_t)bh * (D * D) + (size_t)r * D + ehalf * 64 + zh * 32;
 #pragma unroll
         for (int x = 0; x < 8; ++x)
           *reinterpret_cast<float4*>(dst + 4 * x) = make_float4(zreg[4 * x], zreg[4 * x + 1], zreg[4 * x + 2], zreg[4 * x + 3]);
@@ -702,6 +799,8 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
         tc_fence_after_sync();
         constexpr int PASSES = (sizeof(TOut) == 4) ? 2 : 1;  // 128 bytes of each output row per pass
         constexpr int PIECES = (sizeof(TOut) == 4) ? 2 : 4;  // 16-column accumulator pieces per pass
+        const bool direct = (args.tune & 1) != 0;
+        if (direct && warp == 20 && lane == 0) mbar_arrive(&sm.bars[C_FREE0 + s]);  // M4 was the tile's last reader
 #pragma unroll
         for (int pass = 0; pass < PASSES; ++pass) {
           uint32_t w[32];  // this thread's 128 bytes of the pass
@@ -731,6 +830,17 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
               }
             }
           }
+          if (direct) {
+            // this thread's 128 bytes of row r go straight to global memory as four 32-byte stores (whole
+            // sectors), no staging in shared memory
+            if (r < Cr) {
+              unsigned char* dst = static_cast<unsigned char*>(job.out) +
+                                   (((size_t)bh * args.N + t0 + r) * D + ehalf * 64) * sizeof(TOut) + pass * 128;
+#pragma unroll
+              for (int c = 0; c < 4; ++c) st_global_v8(dst + 32 * c, &w[8 * c]);
+            }
+            continue;
+          }
           if (pass > 0) {
             // the staging tile still feeds the previous pass's store until its source has been read
             if (warp == 20 && lane == 0) tma_store_wait_read();
@@ -749,11 +859,11 @@ tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUte
           ++og_uses;
           if (warp == 20 && lane == 0) {
             // rows beyond N are clipped by the tensor map (a ragged block is always the last of the sequence)
-            tma_store_3d(&tm_out, stg, ehalf * 64 + pass * (int)(128 / sizeof(TOut)), t0, bh);
+            tma_store_3d(tm_out, stg, ehalf * 64 + pass * (int)(128 / sizeof(TOut)), t0, bh);
             tma_store_commit();
           }
         }
-        if (warp == 20 && lane == 0) {
+        if (!direct && warp == 20 && lane == 0) {
           tma_store_wait_read();
           mbar_arrive(&sm.bars[C_FREE0 + s]);  // the c tile of this stage may be reloaded
         }
@@ -830,43 +940,86 @@ bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, int D, bool f32 = 
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool REV, bool STATE_ONLY, typename TOut, int D>
-cudaError_t launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mo,
-                     const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
+// Experiment switches for the tensor-core kernels, from the environment variable LA_TC_TUNE (read once).
+int tune_env() {
+  static const int v = []() {
+    const char* e = getenv("LA_TC_TUNE");
+    return e ? atoi(e) : 4;
+  }();
+  return v;
+}
+
+template <bool REV, bool STATE_ONLY, typename TOut, int D, int NJOBS>
+cudaError_t launch_t(const TcMaps& m0, const TcMaps& m1, const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
   const size_t smem = sizeof(TcSmem) + 1024;
-  auto kern = tc_kernel<REV, STATE_ONLY, TOut, D>;
+  auto kern = tc_kernel<REV, STATE_ONLY, TOut, D, NJOBS>;
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  KernelTimer timer(STATE_ONLY ? K_PREPASS : K_WALK, stream);
-  kern<<<(unsigned)(ta.BH * ta.nseg * (D == 128 ? 2 : 1)), TC_THREADS, smem, stream>>>(ma, mb, mc, mo, ta, tab);
+  KernelTimer timer(STATE_ONLY ? K_PREPASS : (NJOBS == 2 ? K_WALK_PAIR : K_WALK), stream);
+  kern<<<(unsigned)(ta.BH * ta.nseg * (D == 128 ? 2 : 1) * NJOBS), TC_THREADS, smem, stream>>>(m0, m1, ta, tab);
   count_launch();
   return cudaGetLastError();
 }
 
+bool make_maps(TcMaps* m, const OpArgs& args, int D, bool f32) {
+  return make_map(&m->a, args.a, args.N, args.BH, D) && make_map(&m->b, args.b, args.N, args.BH, D) &&
+         make_map(&m->c, args.c, args.N, args.BH, D) && make_map(&m->out, args.out, args.N, args.BH, D, f32);
+}
+
+// One walk (second == nullptr) or two walks of the same direction over the same tokens in one launch.
 template <int D>
-cudaError_t launch_walk_d(const OpArgs& args, const DecayTable& tab, int out_dt, int precision, cudaStream_t stream) {
-  CUtensorMap ma, mb, mc, mo;
+cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayTable& tab, int out_dt, int precision,
+                          cudaStream_t stream) {
+  TcMaps m0, m1;
   const bool f32 = (out_dt == DT_F32);
-  if (!make_map(&ma, args.a, args.N, args.BH, D) || !make_map(&mb, args.b, args.N, args.BH, D) ||
-      !make_map(&mc, args.c, args.N, args.BH, D) || !make_map(&mo, args.out, args.N, args.BH, D, f32))
-    return cudaErrorInvalidValue;
-  TcArgs ta{args.c, args.out, args.entry, nullptr, args.final_out, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
+  if (!make_maps(&m0, args, D, f32)) return cudaErrorInvalidValue;
+  if (second) {
+    if (!make_maps(&m1, *second, D, f32)) return cudaErrorInvalidValue;
+  } else {
+    m1 = m0;
+  }
+  int tune = tune_env();
+  // the direct 32-byte stores need that alignment
+  if ((reinterpret_cast<uintptr_t>(args.out) & 31u) || (second && (reinterpret_cast<uintptr_t>(second->out) & 31u)))
+    tune &= ~1;
+  TcArgs ta{};
+  ta.job[0] = TcJob{args.c, args.out, args.entry, args.final_out};
+  ta.job[1] = second ? TcJob{second->c, second->out, second->entry, second->final_out} : ta.job[0];
+  ta.local_out = nullptr;
+  ta.njobs = second ? 2 : 1;
+  ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
+  ta.precision = precision;
+  ta.tune = tune;
+  if (second) {  // only the reverse direction is ever paired
+    if (!args.reverse) return cudaErrorInvalidValue;
+    return f32 ? launch_t<true, false, float, D, 2>(m0, m1, ta, tab, stream)
+               : launch_t<true, false, __nv_bfloat16, D, 2>(m0, m1, ta, tab, stream);
+  }
   if (args.reverse)
-    return f32 ? launch_t<true, false, float, D>(ma, mb, mc, mo, ta, tab, stream)
-               : launch_t<true, false, __nv_bfloat16, D>(ma, mb, mc, mo, ta, tab, stream);
-  return f32 ? launch_t<false, false, float, D>(ma, mb, mc, mo, ta, tab, stream)
-             : launch_t<false, false, __nv_bfloat16, D>(ma, mb, mc, mo, ta, tab, stream);
+    return f32 ? launch_t<true, false, float, D, 1>(m0, m1, ta, tab, stream)
+               : launch_t<true, false, __nv_bfloat16, D, 1>(m0, m1, ta, tab, stream);
+  return f32 ? launch_t<false, false, float, D, 1>(m0, m1, ta, tab, stream)
+             : launch_t<false, false, __nv_bfloat16, D, 1>(m0, m1, ta, tab, stream);
 }
 
 template <int D>
 cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int precision, cudaStream_t stream) {
-  CUtensorMap mb, mc;
-  if (!make_map(&mb, args.b, args.N, args.BH, D) || !make_map(&mc, args.c, args.N, args.BH, D))
+  TcMaps m;
+  // the a and out maps are unused by the state-only kernel; valid descriptors are passed anyway
+  if (!make_map(&m.b, args.b, args.N, args.BH, D) || !make_map(&m.c, args.c, args.N, args.BH, D))
     return cudaErrorInvalidValue;
-  TcArgs ta{args.c, nullptr, nullptr, args.local_out, nullptr, args.BH, args.H, args.N, args.seg_len, args.nseg, precision};
-  // the a and out maps are unused by the state-only kernel; pass valid descriptors anyway
-  return args.reverse ? launch_t<true, true, float, D>(mb, mb, mc, mc, ta, tab, stream)
-                      : launch_t<false, true, float, D>(mb, mb, mc, mc, ta, tab, stream);
+  m.a = m.b;
+  m.out = m.c;
+  TcArgs ta{};
+  ta.job[0] = TcJob{args.c, nullptr, nullptr, nullptr};
+  ta.job[1] = ta.job[0];
+  ta.local_out = args.local_out;
+  ta.njobs = 1;
+  ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
+  ta.precision = precision;
+  ta.tune = tune_env();
+  return args.reverse ? launch_t<true, true, float, D, 1>(m, m, ta, tab, stream)
+                      : launch_t<false, true, float, D, 1>(m, m, ta, tab, stream);
 }
 
 }  // namespace
@@ -875,8 +1028,19 @@ bool tc_supported() { return encode_fn() != nullptr; }
 
 cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int out_dt, int precision,
                            cudaStream_t stream) {
-  return D == 128 ? launch_walk_d<128>(args, tab, out_dt, precision, stream)
-                  : launch_walk_d<64>(args, tab, out_dt, precision, stream);
+  return D == 128 ? launch_walk_d<128>(args, nullptr, tab, out_dt, precision, stream)
+                  : launch_walk_d<64>(args, nullptr, tab, out_dt, precision, stream);
+}
+
+bool tc_pair_enabled() { return (tune_env() & 2) != 0; }
+
+cudaError_t launch_tc_walk_pair(const OpArgs& first, const OpArgs& second, const DecayTable& tab, int D, int out_dt,
+                                int precision, cudaStream_t stream) {
+  if (first.reverse != second.reverse || first.N != second.N || first.BH != second.BH || first.nseg != second.nseg ||
+      first.seg_len != second.seg_len)
+    return cudaErrorInvalidValue;
+  return D == 128 ? launch_walk_d<128>(first, &second, tab, out_dt, precision, stream)
+                  : launch_walk_d<64>(first, &second, tab, out_dt, precision, stream);
 }
 
 cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, int precision, cudaStream_t stream) {

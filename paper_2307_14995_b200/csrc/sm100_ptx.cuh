@@ -93,6 +93,13 @@ __device__ __forceinline__ void tma_store_wait_read() {
 }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// 32-byte store to global memory (one whole sector; address 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(void* gptr, const uint32_t* w) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(gptr), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+
 // ---- TMEM ----------------------------------------------------------------------------------------
 // One full warp allocates `ncols` (power of two >= 32) columns; the base address lands in *slot.
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot_smem, uint32_t ncols) {
@@ -211,6 +218,83 @@ __device__ __forceinline__ void umma_bf16_lh(uint32_t d_tmem, uint32_t a_lo, uin
       "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(go)
       : "memory");
 }
+// The same with the A operand read from tensor memory.
+__device__ __forceinline__ void umma_bf16_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                                uint32_t idesc, uint32_t accumulate, uint32_t go) {
+  asm volatile(
+      "{\n\t.reg .pred p, g;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 g, %6, 0;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "@g tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(go)
+      : "memory");
+}
+// A whole K loop in one instruction sequence: NK tensor-core instructions D[tmem] (+)= A_k * B_k, k = 0..NK-1,
+// all predicated on `go`, the first one accumulating only if `acc0`.  Operand k is operand 0 moved by a
+// compile-time step: for shared-memory operands the low descriptor half advances by step(k) (16-byte units),
+// AK / BK select the step pattern (true: K-major tile of two 64-element panels 16 KB apart, 32 bytes per K step
+// inside a panel; false: MN-major tile, 2 KB per K step); for a tensor-memory A operand the column advances by
+// 16 per K step.  One predicate set-up for the group instead of one per instruction keeps the issuing warp's
+// instruction count per MMA at three.
+template <bool K_MAJOR>
+__host__ __device__ constexpr uint32_t umma_kstep(int k) {
+  return K_MAJOR ? (uint32_t)((k >> 2) * 1024 + (k & 3) * 2) : (uint32_t)(k * 128);
+}
+#define LA_UMMA_SS_STEP(AI, BI)                                  \
+  "add.u32 al, %1, " #AI ";\n\tmov.b64 da, {al, %3};\n\t"        \
+  "add.u32 bl, %2, " #BI ";\n\tmov.b64 db, {bl, %3};\n\t"        \
+  "@g tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, t;\n\t"
+template <int NK, bool AK, bool BK>
+__device__ __forceinline__ void umma_group_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                              uint32_t idesc, uint32_t acc0, uint32_t go) {
+  static_assert(NK == 4 || NK == 8, "K steps per group");
+  if (NK == 8) {
+    asm volatile(
+        "{\n\t.reg .pred p, g, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 g, %6, 0;\n\tsetp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "@g tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t"
+        LA_UMMA_SS_STEP(%7, %14) LA_UMMA_SS_STEP(%8, %15) LA_UMMA_SS_STEP(%9, %16) LA_UMMA_SS_STEP(%10, %17)
+        LA_UMMA_SS_STEP(%11, %18) LA_UMMA_SS_STEP(%12, %19) LA_UMMA_SS_STEP(%13, %20)
+        "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc0), "r"(go),
+        "n"(umma_kstep<AK>(1)), "n"(umma_kstep<AK>(2)), "n"(umma_kstep<AK>(3)), "n"(umma_kstep<AK>(4)),
+        "n"(umma_kstep<AK>(5)), "n"(umma_kstep<AK>(6)), "n"(umma_kstep<AK>(7)),
+        "n"(umma_kstep<BK>(1)), "n"(umma_kstep<BK>(2)), "n"(umma_kstep<BK>(3)), "n"(umma_kstep<BK>(4)),
+        "n"(umma_kstep<BK>(5)), "n"(umma_kstep<BK>(6)), "n"(umma_kstep<BK>(7))
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p, g, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 g, %6, 0;\n\tsetp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "@g tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t"
+        LA_UMMA_SS_STEP(%7, %10) LA_UMMA_SS_STEP(%8, %11) LA_UMMA_SS_STEP(%9, %12)
+        "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc0), "r"(go),
+        "n"(umma_kstep<AK>(1)), "n"(umma_kstep<AK>(2)), "n"(umma_kstep<AK>(3)),
+        "n"(umma_kstep<BK>(1)), "n"(umma_kstep<BK>(2)), "n"(umma_kstep<BK>(3))
+        : "memory");
+  }
+}
+#undef LA_UMMA_SS_STEP
+// Eight K steps with A in tensor memory (16 columns per step) and an MN-major B tile in shared memory.
+#define LA_UMMA_TS_STEP(AI, BI)                                  \
+  "add.u32 at, %1, " #AI ";\n\t"                                 \
+  "add.u32 bl, %2, " #BI ";\n\tmov.b64 db, {bl, %3};\n\t"        \
+  "@g tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, t;\n\t"
+__device__ __forceinline__ void umma_group_ts8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                               uint32_t idesc, uint32_t acc0, uint32_t go) {
+  asm volatile(
+      "{\n\t.reg .pred p, g, t;\n\t.reg .b64 db;\n\t.reg .b32 at, bl;\n\t"
+      "setp.ne.b32 g, %6, 0;\n\tsetp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "@g tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t"
+      LA_UMMA_TS_STEP(16, 128) LA_UMMA_TS_STEP(32, 256) LA_UMMA_TS_STEP(48, 384) LA_UMMA_TS_STEP(64, 512)
+      LA_UMMA_TS_STEP(80, 640) LA_UMMA_TS_STEP(96, 768) LA_UMMA_TS_STEP(112, 896)
+      "}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc0), "r"(go)
+      : "memory");
+}
+#undef LA_UMMA_TS_STEP
 __device__ __forceinline__ void umma_commit_if(uint64_t* bar, uint32_t go) {
   asm volatile(
       "{\n\t.reg .pred g;\n\tsetp.ne.b32 g, %1, 0;\n\t"
