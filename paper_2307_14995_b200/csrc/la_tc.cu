@@ -909,6 +909,8 @@ __global__ void bounded_wait_selftest_kernel(long long budget) {
   }
 }
 
+#include "la_tc_full.cuh"
+
 // ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -944,7 +946,7 @@ bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, int D, bool f32 = 
 int tune_env() {
   static const int v = []() {
     const char* e = getenv("LA_TC_TUNE");
-    return e ? atoi(e) : 4;
+    return e ? atoi(e) : 12;
   }();
   return v;
 }
@@ -982,6 +984,8 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   // the direct 32-byte stores need that alignment
   if ((reinterpret_cast<uintptr_t>(args.out) & 31u) || (second && (reinterpret_cast<uintptr_t>(second->out) & 31u)))
     tune &= ~1;
+  const int tune_all = tune_env();
+  (void)tune_all;
   TcArgs ta{};
   ta.job[0] = TcJob{args.c, args.out, args.entry, args.final_out};
   ta.job[1] = second ? TcJob{second->c, second->out, second->entry, second->final_out} : ta.job[0];
@@ -990,6 +994,12 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
   ta.tune = tune;
+  if (D == 128 && !second && (tune_env() & 8) && !(reinterpret_cast<uintptr_t>(args.out) & 31u)) {
+    // full-width kernel: one thread block per (head, segment); its 32-byte output stores need that alignment
+    if (args.reverse)
+      return f32 ? launch_full_t<true, float>(m0, ta, tab, stream) : launch_full_t<true, __nv_bfloat16>(m0, ta, tab, stream);
+    return f32 ? launch_full_t<false, float>(m0, ta, tab, stream) : launch_full_t<false, __nv_bfloat16>(m0, ta, tab, stream);
+  }
   if (second) {  // only the reverse direction is ever paired
     if (!args.reverse) return cudaErrorInvalidValue;
     return f32 ? launch_t<true, false, float, D, 2>(m0, m1, ta, tab, stream)
