@@ -309,8 +309,7 @@ def run_ours(args):
                               "ms_per_step_median": ms_median, "ms_per_step_min": ms_min, "clocks": sampler.stop(),
                               "kernel_ms_per_step": {n: ms / prof_steps for n, (ms, _) in prof.items()},
                               "kernel_launches_per_step": {n: c / prof_steps for n, (_, c) in prof.items()},
-                              "walk_gbs": achieved, "walk_pair_gbs": pair_gbs,
-                              "tune": os.environ.get("LA_TC_TUNE")}), flush=True)
+                              "walk_gbs": achieved, "walk_pair_gbs": pair_gbs}), flush=True)
         return
 
     # forward and backward also timed on their own (same buffers, same rules), after the headline loop

@@ -86,7 +86,8 @@ la_status make_plan(const la_shape* s, Plan* p) {
     // time: pick the segment count that minimises (waves over the 148 SMs) x (blocks walked per
     // segment + pipeline fill), with segments no shorter than 1024 tokens so that the
     // per-segment state traffic stays small.  Depends on the shape only.
-    const long slices = (p->tensor && s->d == 128) ? 2 : 1;  // at d = 128 the tensor kernels also split the value columns
+    // at d = 128 the half-width tensor kernels also split the value columns over two thread blocks
+    const long slices = (p->tensor && s->d == 128 && !tc_full_width()) ? 2 : 1;
     const long sms = 148, fill = 2;
     long most = s->N / 1024;
     if (most < 1) most = 1;
@@ -324,7 +325,7 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
     entry_v = buf_e;
     entry_k = buf_et;
   }
-  if (p.tensor && tc_pair_enabled()) {
+  if (p.tensor) {
     // both reverse walks in one launch: together they read Q, K, V and dO, and the thread blocks of the two are
     // interleaved so that each of those tiles comes from HBM once (Algorithm 4 accumulates dK_j and dV_j in the
     // same outer iteration for the same reason)

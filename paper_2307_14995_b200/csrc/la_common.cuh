@@ -79,7 +79,9 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int
                            cudaStream_t stream);
 // Two walks of the same direction over the same tokens (same N, BH, segments) in one launch; the thread blocks of
 // the two are interleaved so that tiles both read come from HBM once.
-bool tc_pair_enabled();
+// Whether the d = 128 walk normally runs as one full-width thread block per (head, segment) rather than two
+// half-width ones (the segment plan counts thread blocks accordingly).
+bool tc_full_width();
 cudaError_t launch_tc_walk_pair(const OpArgs& first, const OpArgs& second, const DecayTable& tab, int D, int out_dt,
                                 int precision, cudaStream_t stream);
 cudaError_t launch_tc_prepass(const OpArgs& args, const DecayTable& tab, int D, int precision,

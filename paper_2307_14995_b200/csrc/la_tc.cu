@@ -54,8 +54,6 @@
 // K-major in M1 and MN-major (as b^T) in M3 from the same bytes.
 #include <cuda.h>
 
-#include <cstdlib>
-
 #include "la_common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -118,7 +116,6 @@ struct TcArgs {
   int njobs;
   int BH, H, N, seg_len, nseg;
   int precision;
-  int tune;  // experiment switches (environment variable LA_TC_TUNE, read once)
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
@@ -386,10 +383,11 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
       }
       umma_commit_if(&sm.bars[DZ_READY], go);
     }
-  } else if (warp == 1 && (args.tune & 4)) {
-    // ------------------------------------ MMA issuer, walk kernel, warp-convergent form ------------------------------------
-    // The same schedule as the single-lane form below, run by all 32 lanes together; only the tensor-core
-    // instructions and their commits are predicated on one elected lane.
+  } else if (warp == 1) {
+    // ------------------------------------ MMA issuer, walk kernel ------------------------------------
+    // All 32 lanes run this loop converged (waits included); the tensor-core instructions and their commits take
+    // effect in one elected lane only, a whole K loop per instruction sequence (measured: 4 % faster than issuing
+    // from inside an `if (lane == 0)` region).
     {
       constexpr uint32_t ID_S = umma_idesc_bf16(128, 128, false, false);
       constexpr uint32_t ID_KN = umma_idesc_bf16(128, 64, false, true);
@@ -438,103 +436,6 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
         umma_group_ts8(tmem + COL_OI, tmem + col_p, cms, HI, ID_KN, 0, go);
         if (split_p) umma_group_ts8(tmem + COL_OI, tmem + col_p + 8, cms, HI, ID_KN, 1, go);
         umma_commit_if(&sm.bars[O_READY], go);
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------ MMA issuer, walk kernel ------------------------------------
-    if (lane == 0) {
-      mma_elected = 1;
-      constexpr uint32_t ID_S = umma_idesc_bf16(128, 128, false, false);   // a (K-major) x b (K-major)
-      constexpr uint32_t ID_KN = umma_idesc_bf16(128, 64, false, true);    // K-major A x MN-major B, N = 64
-      constexpr uint32_t ID_MN64 = umma_idesc_bf16(128, 64, true, true);   // b^T (MN-major A) x MN-major B
-      const uint32_t zh0 = smem_u32(&sm.z_hi[0]), zl0 = smem_u32(&sm.z_lo[0]);
-      const uint32_t fh0 = smem_u32(&sm.fc_hi[0]);
-      {
-        // prologue: S(0)
-        {
-          const uint32_t a0 = smem_u32(&sm.st[0].a[0][0]), b0 = smem_u32(&sm.st[0].b[0][0]);
-          TC_WAIT(FULL_B0, 0, 7);  // a and b of block 0
-          tc_fence_after_sync();
-#pragma unroll
-          for (int k = 0; k < KD; ++k) {
-            const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
-            umma_bf16(tmem + COL_S0, umma_desc_sw128(a0 + ko, 16, 1024), umma_desc_sw128(b0 + ko, 16, 1024), ID_S,
-                      k > 0);
-          }
-          issued_mma = true;
-          umma_commit(&sm.bars[S_READY0]);
-        }
-        for (int it = 0; it < nblk; ++it) {
-          const int s = it & 1;
-          const uint32_t par1 = it & 1, par2 = (it >> 1) & 1;
-          const uint32_t a0 = smem_u32(&sm.st[s].a[0][0]), b0 = smem_u32(&sm.st[s].b[0][0]);
-          const uint32_t c0 = smem_u32(&sm.st[s].c[0]);
-          const uint32_t col_p = s ? COL_S1 : COL_S0;
-          // M3: dZ = b^T [fc_hi | fc_lo]  (needs the previous dZ to have been read)
-          // Z_READY: the state operand of this block AND fc of this block are in place (the Z group forms fc first)
-          TC_WAIT(Z_READY, par1, 12);
-          tc_fence_after_sync();
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_bf16(tmem + COL_DZ, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
-                      umma_desc_sw128(fh0 + k * 2048, 16384, 1024), ID_MN64, k > 0);
-          if (split_c) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              umma_bf16(tmem + COL_DZ, umma_desc_sw128(b0 + k * 2048, 16384, 1024),
-                        umma_desc_sw128(fh0 + 16384 + k * 2048, 16384, 1024), ID_MN64, 1);
-          }
-          umma_commit(&sm.bars[DZ_READY]);
-          // M2: O_inter = a Z   (state after the previous block / the entry state)
-          // this O_inter buffer was last read for block it-2; that read was already awaited before M4(it-1)
-          const uint32_t col_oe = (it & 1) ? COL_OE1 : COL_OE0;
-          tc_fence_after_sync();
-#pragma unroll
-          for (int k = 0; k < KD; ++k) {
-            const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
-            umma_bf16(tmem + col_oe, umma_desc_sw128(a0 + ko, 16, 1024),
-                      umma_desc_sw128(zh0 + k * 2048, 16384, 1024), ID_KN, k > 0);
-          }
-          if (split_z) {
-#pragma unroll
-            for (int k = 0; k < KD; ++k) {
-              const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
-              umma_bf16(tmem + col_oe, umma_desc_sw128(a0 + ko, 16, 1024),
-                        umma_desc_sw128(zl0 + k * 2048, 16384, 1024), ID_KN, 1);
-            }
-          }
-          umma_commit(&sm.bars[A_FREE0 + s]);  // M1 and M2 of this block are done with the a tile
-          // M1 of the next block, into the other S/P buffer
-          if (it + 1 < nblk) {
-            const int s1 = s ^ 1;
-            const uint32_t parn = ((it + 1) >> 1) & 1;
-            const uint32_t an = smem_u32(&sm.st[s1].a[0][0]), bn = smem_u32(&sm.st[s1].b[0][0]);
-            TC_WAIT(FULL_B0 + s1, parn, 11);  // a and b of the next block
-            tc_fence_after_sync();
-#pragma unroll
-            for (int k = 0; k < KD; ++k) {
-              const uint32_t ko = (k >> 2) * 16384 + (k & 3) * 32;
-              umma_bf16(tmem + (s1 ? COL_S1 : COL_S0), umma_desc_sw128(an + ko, 16, 1024),
-                        umma_desc_sw128(bn + ko, 16, 1024), ID_S, k > 0);
-            }
-            umma_commit(&sm.bars[S_READY0 + s1]);
-          }
-          // M4: O_intra = P c, P read from tensor memory (K step k: hi pairs at column 16k, lo pairs at 16k+8)
-          TC_WAIT(P_READY0 + s, par2, 14);  // P is written and the accumulators of the previous block have been read
-          TC_WAIT(FULL_C0 + s, par2, 15);
-          tc_fence_after_sync();
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_bf16_ts(tmem + COL_OI, tmem + col_p + 16 * k, umma_desc_sw128(c0 + k * 2048, 16384, 1024), ID_KN,
-                         k > 0);
-          if (split_p) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              umma_bf16_ts(tmem + COL_OI, tmem + col_p + 16 * k + 8, umma_desc_sw128(c0 + k * 2048, 16384, 1024),
-                           ID_KN, 1);
-          }
-          umma_commit(&sm.bars[O_READY]);
-        }
       }
     }
   } else if (STATE_ONLY && warp >= 4 && warp < 20) {
@@ -799,8 +700,6 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
         tc_fence_after_sync();
         constexpr int PASSES = (sizeof(TOut) == 4) ? 2 : 1;  // 128 bytes of each output row per pass
         constexpr int PIECES = (sizeof(TOut) == 4) ? 2 : 4;  // 16-column accumulator pieces per pass
-        const bool direct = (args.tune & 1) != 0;
-        if (direct && warp == 20 && lane == 0) mbar_arrive(&sm.bars[C_FREE0 + s]);  // M4 was the tile's last reader
 #pragma unroll
         for (int pass = 0; pass < PASSES; ++pass) {
           uint32_t w[32];  // this thread's 128 bytes of the pass
@@ -830,17 +729,6 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
               }
             }
           }
-          if (direct) {
-            // this thread's 128 bytes of row r go straight to global memory as four 32-byte stores (whole
-            // sectors), no staging in shared memory
-            if (r < Cr) {
-              unsigned char* dst = static_cast<unsigned char*>(job.out) +
-                                   (((size_t)bh * args.N + t0 + r) * D + ehalf * 64) * sizeof(TOut) + pass * 128;
-#pragma unroll
-              for (int c = 0; c < 4; ++c) st_global_v8(dst + 32 * c, &w[8 * c]);
-            }
-            continue;
-          }
           if (pass > 0) {
             // the staging tile still feeds the previous pass's store until its source has been read
             if (warp == 20 && lane == 0) tma_store_wait_read();
@@ -863,7 +751,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
             tma_store_commit();
           }
         }
-        if (!direct && warp == 20 && lane == 0) {
+        if (warp == 20 && lane == 0) {
           tma_store_wait_read();
           mbar_arrive(&sm.bars[C_FREE0 + s]);  // the c tile of this stage may be reloaded
         }
@@ -942,15 +830,6 @@ bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, int D, bool f32 = 
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Experiment switches for the tensor-core kernels, from the environment variable LA_TC_TUNE (read once).
-int tune_env() {
-  static const int v = []() {
-    const char* e = getenv("LA_TC_TUNE");
-    return e ? atoi(e) : 12;
-  }();
-  return v;
-}
-
 template <bool REV, bool STATE_ONLY, typename TOut, int D, int NJOBS>
 cudaError_t launch_t(const TcMaps& m0, const TcMaps& m1, const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
   const size_t smem = sizeof(TcSmem) + 1024;
@@ -980,12 +859,6 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   } else {
     m1 = m0;
   }
-  int tune = tune_env();
-  // the direct 32-byte stores need that alignment
-  if ((reinterpret_cast<uintptr_t>(args.out) & 31u) || (second && (reinterpret_cast<uintptr_t>(second->out) & 31u)))
-    tune &= ~1;
-  const int tune_all = tune_env();
-  (void)tune_all;
   TcArgs ta{};
   ta.job[0] = TcJob{args.c, args.out, args.entry, args.final_out};
   ta.job[1] = second ? TcJob{second->c, second->out, second->entry, second->final_out} : ta.job[0];
@@ -993,12 +866,20 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   ta.njobs = second ? 2 : 1;
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
-  ta.tune = tune;
-  if (D == 128 && !second && (tune_env() & 8) && !(reinterpret_cast<uintptr_t>(args.out) & 31u)) {
-    // full-width kernel: one thread block per (head, segment); its 32-byte output stores need that alignment
+  if (D == 128 && !(reinterpret_cast<uintptr_t>(args.out) & 31u) &&
+      !(second && (reinterpret_cast<uintptr_t>(second->out) & 31u))) {
+    // full-width kernel: one thread block per (head, segment).  Its 32-byte output stores need that alignment;
+    // an output that is only 16-byte aligned (the contract's minimum) takes the half-width kernels below.
+    if (second) {
+      if (!args.reverse) return cudaErrorInvalidValue;
+      return f32 ? launch_full_t<true, float, 2>(m0, m1, ta, tab, stream)
+                 : launch_full_t<true, __nv_bfloat16, 2>(m0, m1, ta, tab, stream);
+    }
     if (args.reverse)
-      return f32 ? launch_full_t<true, float>(m0, ta, tab, stream) : launch_full_t<true, __nv_bfloat16>(m0, ta, tab, stream);
-    return f32 ? launch_full_t<false, float>(m0, ta, tab, stream) : launch_full_t<false, __nv_bfloat16>(m0, ta, tab, stream);
+      return f32 ? launch_full_t<true, float, 1>(m0, m1, ta, tab, stream)
+                 : launch_full_t<true, __nv_bfloat16, 1>(m0, m1, ta, tab, stream);
+    return f32 ? launch_full_t<false, float, 1>(m0, m1, ta, tab, stream)
+               : launch_full_t<false, __nv_bfloat16, 1>(m0, m1, ta, tab, stream);
   }
   if (second) {  // only the reverse direction is ever paired
     if (!args.reverse) return cudaErrorInvalidValue;
@@ -1027,7 +908,6 @@ cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int prec
   ta.njobs = 1;
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
-  ta.tune = tune_env();
   return args.reverse ? launch_t<true, true, float, D, 1>(m, m, ta, tab, stream)
                       : launch_t<false, true, float, D, 1>(m, m, ta, tab, stream);
 }
@@ -1042,7 +922,7 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int
                   : launch_walk_d<64>(args, nullptr, tab, out_dt, precision, stream);
 }
 
-bool tc_pair_enabled() { return (tune_env() & 2) != 0; }
+bool tc_full_width() { return true; }
 
 cudaError_t launch_tc_walk_pair(const OpArgs& first, const OpArgs& second, const DecayTable& tab, int D, int out_dt,
                                 int precision, cudaStream_t stream) {

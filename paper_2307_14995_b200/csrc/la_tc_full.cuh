@@ -66,15 +66,23 @@ __device__ __forceinline__ void reg_inc() {
   asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
-template <bool REV, typename TOut>
+// NJOBS = 2: two walks of the same direction over the same tokens in one launch (the dV and dK walks of the backward
+// pass, which between them read Q, K, V and dO); the thread blocks of the two jobs alternate, so that the two
+// readers of a tile run side by side and the tile comes from HBM once.
+template <bool REV, typename TOut, int NJOBS>
 __global__ void __launch_bounds__(F_THREADS, 1)
-tc_walk_full_kernel(const __grid_constant__ TcMaps maps, const TcArgs args, const DecayTable tab) {
+tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps maps1, const TcArgs args,
+                    const DecayTable tab) {
   extern __shared__ unsigned char smem_raw[];
   FSmem& sm = *reinterpret_cast<FSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const TcJob job = args.job[0];
-  const int bh = (int)blockIdx.x / args.nseg, seg = (int)blockIdx.x % args.nseg;
+  const int jobid = (NJOBS == 2) ? (int)(blockIdx.x & 1) : 0;
+  const int bidx = (NJOBS == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  TcJob job = args.job[0];
+  if (NJOBS == 2 && jobid) job = args.job[1];
+  const TcMaps& maps = (NJOBS == 2 && jobid) ? maps1 : maps0;
+  const int bh = bidx / args.nseg, seg = bidx % args.nseg;
   const int seg_t0 = seg * args.seg_len;
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
   const int nblk = (seg_t1 - seg_t0 + 127) >> 7;
@@ -242,7 +250,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps, const TcArgs args, cons
       const int t0 = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;
       const int Cr = min(128, seg_t1 - t0);
       if (r >= Cr) return 0.f;
-      return REV ? exp2f(-s2 * (float)(r + 1)) : exp2f(-s2 * (float)(Cr - 1 - r));
+      return REV ? ex2_approx(-s2 * (float)(r + 1)) : ex2_approx(-s2 * (float)(Cr - 1 - r));
     };
     // fc = diag(f_state) c for this warp's 32 columns of row r
     auto make_fc = [&](const uint4 (&raw)[4], float f) {
@@ -318,7 +326,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps, const TcArgs args, cons
         TC_WAIT_WARP(F_DZ_READY, it & 1, 22);
         tc_fence_after_sync();
         {
-          const float gamma = exp2f(-s2 * (float)Cr);
+          const float gamma = ex2_approx(-s2 * (float)Cr);
 #pragma unroll
           for (int pc = 0; pc < 2; ++pc) {
             uint32_t dh[16];
@@ -368,7 +376,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps, const TcArgs args, cons
       const int t0 = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;
       const int Cr = min(128, seg_t1 - t0);
       float f = 0.f;
-      if (r < Cr) f = REV ? exp2f(-s2 * (float)(Cr - 1 - r)) : exp2f(-s2 * (float)(r + 1));
+      if (r < Cr) f = REV ? ex2_approx(-s2 * (float)(Cr - 1 - r)) : ex2_approx(-s2 * (float)(r + 1));
       // byte address of column 32 g / 4 .. of this thread's own row; the other rows of the quad are 512 or 256 bytes apart
       unsigned char* const quad_base =
           static_cast<unsigned char*>(job.out) + ((size_t)bh * args.N + t0 + (r & ~3)) * 128 * sizeof(TOut) + g * 32;
@@ -454,14 +462,14 @@ teardown:
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-template <bool REV, typename TOut>
-cudaError_t launch_full_t(const TcMaps& m, const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
+template <bool REV, typename TOut, int NJOBS>
+cudaError_t launch_full_t(const TcMaps& m0, const TcMaps& m1, const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
   const size_t smem = sizeof(FSmem) + 1024;
-  auto kern = tc_walk_full_kernel<REV, TOut>;
+  auto kern = tc_walk_full_kernel<REV, TOut, NJOBS>;
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  KernelTimer timer(K_WALK, stream);
-  kern<<<(unsigned)(ta.BH * ta.nseg), F_THREADS, smem, stream>>>(m, ta, tab);
+  KernelTimer timer(NJOBS == 2 ? K_WALK_PAIR : K_WALK, stream);
+  kern<<<(unsigned)(ta.BH * ta.nseg * NJOBS), F_THREADS, smem, stream>>>(m0, m1, ta, tab);
   count_launch();
   return cudaGetLastError();
 }

@@ -406,6 +406,31 @@ def test_guard_bands_untouched(path, d):
     assert_close(views[0], ref[0], TOL_BF16, "o")
 
 
+def test_outputs_aligned_to_16_bytes_only():
+    """The contract asks for 16-byte alignment.  At d = 128 the full-width kernel stores 32 bytes at a time, so
+    outputs that are 16- but not 32-byte aligned take the half-width kernels: same results."""
+    B, H, N, d = 1, 3, 700, 128
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=33)
+    lam = torch.tensor([1.0, 0.95, 0.4])
+    kv_in = inputs.make_state(B, H, d, d, seed=34)
+    gko = inputs.make_state(B, H, d, d, seed=35)
+    qg, kg, vg, dog, kin, gk = to_dev(q, k, v, do, kv_in, gko)
+    n = B * H * N * d
+    bufs = [torch.zeros(n + 8, dtype=torch.float32, device=DEV) for _ in range(4)]
+    views = [b[4:4 + n].view(B, H, N, d) for b in bufs]  # 16 bytes past a 256-byte aligned base
+    assert all(v_.data_ptr() % 32 == 16 for v_ in views)
+    kv_out, gin = (torch.empty((B, H, d, d), dtype=torch.float32, device=DEV) for _ in range(2))
+    shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, 256)
+    ws_f = la.alloc_workspace(la.LA_OP_FWD, shape, DEV)
+    ws_b = la.alloc_workspace(la.LA_OP_BWD, shape, DEV)
+    la.la_fwd(shape, qg, kg, vg, lam, views[0], kin, kv_out, ws_f)
+    la.la_bwd(shape, qg, kg, vg, dog, lam, views[1], views[2], views[3], kin, gk, gin, ws_b, fwd_workspace=ws_f)
+    torch.cuda.synchronize()
+    la.device_status()
+    ref = oracle_all(q, k, v, do, lam, kv_in.double().numpy(), gko.double().numpy())
+    compare_all((views[0], kv_out, views[1], views[2], views[3], gin), ref, TOL_BF16)
+
+
 @pytest.mark.parametrize("d", [64, 128])
 @pytest.mark.parametrize("path", PATHS)
 def test_causality_bitwise(path, d):
