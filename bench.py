@@ -236,11 +236,12 @@ def run_ours(args):
     data = inputs.device_randn_like_workload(WORKLOAD, dev, seed=rank)
     q, k, v, do, lam = data["q"], data["k"], data["v"], data["do"], data["lam"]
     if args.small:
-        # profiling case: 8 heads x 16384 tokens (inputs + outputs still exceed L2), same kernels
+        # profiling case: 16 heads x 32768 tokens (1.6 GB of inputs and outputs, far beyond L2; one wave of 144
+        # thread blocks of 29 blocks each), same kernels
         import dataclasses
-        w = dataclasses.replace(w, H=8, N=16384)
-        q, k, v, do = (x[:, :8, :16384].contiguous() for x in (q, k, v, do))
-        lam = lam[:8].contiguous()
+        w = dataclasses.replace(w, H=16, N=32768)
+        q, k, v, do = (x[:, :16, :32768].contiguous() for x in (q, k, v, do))
+        lam = lam[:16].contiguous()
     shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype, precision=args.precision)
     o = torch.empty((w.B, w.H, w.N, w.e), dtype=out_dtype, device=dev)
     dq, dk, dv = (torch.empty((w.B, w.H, w.N, w.d), dtype=out_dtype, device=dev) for _ in range(3))
@@ -527,7 +528,7 @@ def main():
     ap.add_argument("--only", default="all", choices=["all", "train", "decode"],
                     help="profiling aid: run only the fwd+bwd leg or only the decode leg (prints a short line)")
     ap.add_argument("--small", action="store_true",
-                    help="profiling aid: 8 heads x 16384 tokens of the workload for the fwd+bwd leg")
+                    help="profiling aid: 16 heads x 32768 tokens of the workload for the fwd+bwd leg")
     ap.add_argument("--decode-steps", type=int, default=0, help="profiling aid: recurrent steps per pass")
     ap.add_argument("--precision", type=int, default=-1,
                     help="experiment: LA_SPLIT_* bits for the tensor-core kernels (-1 = library default, all on; "

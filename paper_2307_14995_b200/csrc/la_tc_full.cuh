@@ -217,12 +217,18 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
 #pragma unroll
             for (int x = 0; x < 16; ++x) d[x] = ex2_approx(-s2 * (REV ? n0 + (float)x : n0 - (float)x));
             tmem_ld_wait();
+            if (REV ? (cc > q) : (cc < q)) {
+              // 32x32 sub-tile wholly inside the causal band: nothing to mask
 #pragma unroll
-            for (int x = 0; x < 16; ++x) {
-              const int j = cc * 32 + hh * 16 + x;
-              const int n = REV ? (j - r) : (r - j);
-              // a select, not a multiply by zero: masked-out tokens can never leak
-              d[x] = (n >= 0) ? __uint_as_float(sreg[x]) * d[x] : 0.f;
+              for (int x = 0; x < 16; ++x) d[x] = __uint_as_float(sreg[x]) * d[x];
+            } else {
+#pragma unroll
+              for (int x = 0; x < 16; ++x) {
+                const int j = cc * 32 + hh * 16 + x;
+                const int n = REV ? (j - r) : (r - j);
+                // a select, not a multiply by zero: masked-out tokens can never leak
+                d[x] = (n >= 0) ? __uint_as_float(sreg[x]) * d[x] : 0.f;
+              }
             }
             split16(d, h8, l8);
           }
