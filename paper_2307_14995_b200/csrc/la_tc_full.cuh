@@ -252,17 +252,24 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
     const int off_base = (cg >> 1) * (128 * 64) + r * 64;
     const int chunk0 = 4 * (cg & 1);
 
-    auto state_factor = [&](int it) -> float {
+    // fc = diag(f_state) c is formed 16 bytes (8 columns) at a time: piece i of this thread is chunk (zt & 15) of
+    // token row 32 i + (zt >> 4), so a warp reads two whole rows of c (512 contiguous bytes) per load instruction
+    // and writes whole 128-byte rows of the operand tile -- row-per-thread loads would touch 32 lines each.
+    const int zt = (warp - 12) * 32 + lane;  // 0 .. 511
+    const int frow = zt >> 4, fch = zt & 15;
+    // decay factor of token row `row` of block iteration `it` in the state update
+    auto state_factor = [&](int it, int row) -> float {
       const int t0 = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;
       const int Cr = min(128, seg_t1 - t0);
-      if (r >= Cr) return 0.f;
-      return REV ? ex2_approx(-s2 * (float)(r + 1)) : ex2_approx(-s2 * (float)(Cr - 1 - r));
+      if (row >= Cr) return 0.f;
+      return REV ? ex2_approx(-s2 * (float)(row + 1)) : ex2_approx(-s2 * (float)(Cr - 1 - row));
     };
-    // fc = diag(f_state) c for this warp's 32 columns of row r
-    auto make_fc = [&](const uint4 (&raw)[4], float f) {
+    auto make_fc = [&](const uint4 (&raw)[4], int it) {
 #pragma unroll
-      for (int x4 = 0; x4 < 4; ++x4) {
-        const uint32_t w[4] = {raw[x4].x, raw[x4].y, raw[x4].z, raw[x4].w};
+      for (int i = 0; i < 4; ++i) {
+        const int row = 32 * i + frow;
+        const float f = state_factor(it, row);
+        const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
         float x8[8];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -272,23 +279,22 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
         }
         uint4 h, l;
         split8(x8, h, l);
-        const int off = off_base + (((chunk0 + x4) ^ (r & 7)) << 3);
+        // MN-major operand tile: two 64-column chunks of 16 KB, rows of 128 bytes, 16-byte units swizzled by row
+        const int off = (fch >> 3) * (128 * 64) + row * 64 + (((fch & 7) ^ (row & 7)) << 3);
         *reinterpret_cast<uint4*>(&sm.fc_hi[0][0] + off) = h;
         if (split_c) *reinterpret_cast<uint4*>(&sm.fc_lo[0][0] + off) = l;
       }
       fence_proxy_async_smem();
     };
-    // this thread's row slice of c straight from global memory; rows beyond N read as zero
+    // this thread's four pieces of c straight from global memory; rows beyond N read as zero
     auto c_from_global = [&](int it, uint4 (&raw)[4]) {
-      const int t = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128 + r;
-      if (t < args.N) {
-        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
-                                                          ((size_t)bh * args.N + t) * 128 + cg * 32);
+      const int t0 = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;
+      const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
+                                                        ((size_t)bh * args.N + t0 + frow) * 128) + fch;
 #pragma unroll
-        for (int x = 0; x < 4; ++x) raw[x] = __ldg(src + x);
-      } else {
-#pragma unroll
-        for (int x = 0; x < 4; ++x) raw[x] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = 0; i < 4; ++i) {
+        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(src + (size_t)i * 32 * 16);  // 32 rows of 16 chunks on
+        else raw[i] = make_uint4(0u, 0u, 0u, 0u);
       }
     };
     {
@@ -321,7 +327,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
       };
       uint4 cnext[4];  // row slice of the next block's c, fetched one block ahead
       c_from_global(0, cnext);
-      make_fc(cnext, state_factor(0));
+      make_fc(cnext, 0);
       if (nblk > 1) c_from_global(1, cnext);
       write_state_operand();
       WARP_ARRIVE(F_Z_READY);
@@ -345,7 +351,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
         }
         if (it + 1 < nblk) {
           // DZ_READY also says M3 of this block is done, so the fc buffer may be rewritten
-          make_fc(cnext, state_factor(it + 1));
+          make_fc(cnext, it + 1);
           if (it + 2 < nblk) c_from_global(it + 2, cnext);
           // M2 of this block is done: it has read the old state operand
           TC_WAIT_WARP(F_AB_FREE, it & 1, 23);
