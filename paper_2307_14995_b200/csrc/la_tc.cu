@@ -561,20 +561,27 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
     const int r = q * 32 + lane;      // token row j of c / state row k of Z
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
 
-    // Decay factor of row r of block iteration `it` in the state update.
-    auto state_factor = [&](int it) -> float {
+    // fc = diag(f_state) c is formed 16 bytes (8 columns) at a time: piece i of this thread is chunk (zt & 7) of
+    // token row 32 i + (zt >> 3), so a warp reads whole 128-byte lines of c per load instruction (four rows of this
+    // block's 64 value columns) and writes whole rows of the operand tile; row-per-thread loads would touch 32
+    // lines per instruction, and the load/store unit's time per line is what every group's shared-memory traffic
+    // then waits behind (measured on the full-width kernel: 7 % of a step).
+    const int zt = (warp - 12) * 32 + lane;  // 0 .. 255
+    const int frow = zt >> 3, fch = zt & 7;
+    // decay factor of token row `row` of block iteration `it` in the state update
+    auto state_factor = [&](int it, int row) -> float {
       const int blk = REV ? (nblk - 1 - it) : it;
       const int t0 = seg_t0 + blk * 128;
       const int Cr = min(128, seg_t1 - t0);
-      if (r >= Cr) return 0.f;
-      return REV ? exp2f(-s2 * (float)(r + 1)) : exp2f(-s2 * (float)(Cr - 1 - r));
+      if (row >= Cr) return 0.f;
+      return REV ? exp2f(-s2 * (float)(row + 1)) : exp2f(-s2 * (float)(Cr - 1 - row));
     };
-    // fc = diag(f_state) c for this warp's 32 columns of row r, given as 4 x 8 raw bf16 (chunks
-    // 4*zh .. 4*zh+3 of the 64-column row), into the swizzled operand buffer at hi_tile / lo_tile.
-    auto make_fc = [&](const uint4 (&raw)[4], float f, __nv_bfloat16* hi_tile, __nv_bfloat16* lo_tile) {
+    auto make_fc = [&](const uint4 (&raw)[4], int it, __nv_bfloat16* hi_tile, __nv_bfloat16* lo_tile) {
 #pragma unroll
-      for (int x4 = 0; x4 < 4; ++x4) {  // 8 elements (one 16-byte chunk) per pass: few live registers
-        const uint32_t w[4] = {raw[x4].x, raw[x4].y, raw[x4].z, raw[x4].w};
+      for (int i = 0; i < 4; ++i) {
+        const int row = 32 * i + frow;
+        const float f = state_factor(it, row);
+        const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
         float x8[8];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -584,25 +591,23 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
         }
         uint4 h, l;
         split8(x8, h, l);
-        const int off = r * 64 + (((4 * zh + x4) ^ (r & 7)) << 3);
+        const int off = row * 64 + ((fch ^ (row & 7)) << 3);
         *reinterpret_cast<uint4*>(hi_tile + off) = h;
         if (split_c) *reinterpret_cast<uint4*>(lo_tile + off) = l;
       }
       fence_proxy_async_smem();
     };
-    // this thread's row slice of c straight from global memory (keeps the shared c tile off the state
-    // chain, so that tile only has to arrive in time for M4); rows beyond N read as zero
+    // this thread's four pieces of c straight from global memory (keeps the shared c tile off the state chain, so
+    // that tile only has to arrive in time for M4); rows beyond N read as zero
     auto c_from_global = [&](int it, uint4 (&raw)[4]) {
       const int blk = REV ? (nblk - 1 - it) : it;
-      const int t = seg_t0 + blk * 128 + r;
-      if (t < args.N) {
-        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
-                                                          ((size_t)bh * args.N + t) * D + ehalf * 64 + zh * 32);
+      const int t0 = seg_t0 + blk * 128;
+      const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
+                                                        ((size_t)bh * args.N + t0 + frow) * D + ehalf * 64) + fch;
 #pragma unroll
-        for (int x = 0; x < 4; ++x) raw[x] = __ldg(src + x);
-      } else {
-#pragma unroll
-        for (int x = 0; x < 4; ++x) raw[x] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = 0; i < 4; ++i) {
+        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(src + (size_t)i * 32 * (D / 8));  // 32 rows of D / 8 chunks on
+        else raw[i] = make_uint4(0u, 0u, 0u, 0u);
       }
     };
 
@@ -637,7 +642,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
       };
       uint4 cnext[4];  // row slice of the next block's c, fetched one block ahead
       c_from_global(0, cnext);
-      make_fc(cnext, state_factor(0), sm.fc_hi, sm.fc_lo);
+      make_fc(cnext, 0, sm.fc_hi, sm.fc_lo);
       if (nblk > 1) c_from_global(1, cnext);
       write_state_operand();
       WARP_ARRIVE(Z_READY);
@@ -662,7 +667,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
         }
         if (it + 1 < nblk) {
           // DZ_READY also says M3 of this block is done, so the fc buffer may be rewritten
-          make_fc(cnext, state_factor(it + 1), sm.fc_hi, sm.fc_lo);
+          make_fc(cnext, it + 1, sm.fc_hi, sm.fc_lo);
           if (it + 2 < nblk) c_from_global(it + 2, cnext);
           // A_FREE of this block's stage: M2 of this block is done, so it has read the old state operand
           TC_WAIT_WARP(A_FREE0 + (it & 1), (it >> 1) & 1, 23);
