@@ -66,11 +66,11 @@ def bytes_per_token_head(d: int, out_bytes: int, what: str) -> float:
 
 
 # DRAM traffic of one walk launch per token-head, from the ncu capture summarised in
-# profiles/tc_walk_kernel_small_case.md: 105.46 MB read per 131072 token-heads (the algorithmic
-# 768 B plus 5 % for entry states and re-fetches).  The writes of that small launch (32 MB of the
-# 67 MB of output; the rest was still in L2 when it ended) do not grow in proportion: at full size
+# profiles/tc_walk_full_kernel_small_case.md: 412.4 MB read per 524288 token-heads (the algorithmic
+# 768 B plus 2.4 % for entry states and re-fetches).  The writes of that small launch (230 MB of the
+# 268 MB of output; the rest was still in L2 when it ended) do not grow in proportion: at full size
 # the 4.3 GB of output cannot stay in the 126 MB L2, so the output is counted in full (512 B).
-WALK_DRAM_BYTES_PER_TOKEN_HEAD = 105.46e6 / 131072 + 512.0
+WALK_DRAM_BYTES_PER_TOKEN_HEAD = 412.4e6 / 524288 + 512.0
 
 
 def load_peaks():
@@ -242,7 +242,7 @@ def run_ours(args):
         w = dataclasses.replace(w, H=16, N=32768)
         q, k, v, do = (x[:, :16, :32768].contiguous() for x in (q, k, v, do))
         lam = lam[:16].contiguous()
-    shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype, precision=args.precision)
+    shape = la.make_shape(w.B, w.H, w.N, w.d, w.e, w.in_dtype, out_dtype, seg_len=args.seg_len, precision=args.precision)
     o = torch.empty((w.B, w.H, w.N, w.e), dtype=out_dtype, device=dev)
     dq, dk, dv = (torch.empty((w.B, w.H, w.N, w.d), dtype=out_dtype, device=dev) for _ in range(3))
     ws_f = la.alloc_workspace(la.LA_OP_FWD, shape, dev)
@@ -459,7 +459,7 @@ def run_ours(args):
                         "bound": ("latency (a few short launches over a shape that fits L2)"
                                   if ow.token_heads < 200000 else "hbm"),
                         "kernels": ("fp32 CUDA cores" if ow.in_dtype == torch.float32 else
-                                    "tcgen05 (one thread block per head and segment at d = 64, two at d = 128)")}
+                                    "tcgen05 (one thread block per head and segment)")}
         del od_, oo, odq, odk, odv, owf, owb, flush
 
     clocks = sampler.stop() if rank == 0 else None
@@ -489,11 +489,11 @@ def run_ours(args):
             "kernel_launches_per_step": {kname: c / prof_steps for kname, (_, c) in prof.items()},
             "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"),
             "roofline": {"scope": "ONE kernel, the dominant one; the whole-step figure the target is stated on is step_roofline",
-                         "kernel": "block walk (tc_kernel, not state-only), single-job launches (O and dQ)", "bound": "hbm",
+                         "kernel": "full-width block walk (tc_walk_full_kernel), single-job launches (O and dQ)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
                          "traffic": WALK_DRAM_BYTES_PER_TOKEN_HEAD * th,
-                         "traffic_note": "ncu dram read bytes of a 131072-token-head launch scaled by token-heads + the full fp32 output",
+                         "traffic_note": "ncu dram read bytes of a 524288-token-head launch scaled by token-heads + the full fp32 output",
                          "peak_source": peaks["source"],
                          "avg_launch_ms": walk_avg_ms, "launches": walk_n, "bytes_per_launch": walk_bytes,
                          "walk_pair": {"what": "the dV and dK walks of the backward pass in one launch",
@@ -530,6 +530,8 @@ def main():
     ap.add_argument("--small", action="store_true",
                     help="profiling aid: 16 heads x 32768 tokens of the workload for the fwd+bwd leg")
     ap.add_argument("--decode-steps", type=int, default=0, help="profiling aid: recurrent steps per pass")
+    ap.add_argument("--seg-len", type=int, default=0,
+                    help="experiment: segment length in tokens (multiple of 128) instead of the library's choice")
     ap.add_argument("--precision", type=int, default=-1,
                     help="experiment: LA_SPLIT_* bits for the tensor-core kernels (-1 = library default, all on; "
                          "anything else does not meet the parity tolerance on every head)")
