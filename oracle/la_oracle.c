@@ -15,6 +15,9 @@
  *       kv_t = lambda kv_{t-1} + k_t v_t^T,   o_t = kv_t^T q_t,   kv_0 = 0
  *   prescaled recurrence (Algorithm 1, "Origin Inference"), kept only to show
  *       where it loses precision and overflows.
+ *   normalisation and gate that follow the attention product in the token mixer
+ *       (Eq. 3 "Gated Linear Attention" with Eq. 8 "SimpleRMSNorm"), per row of
+ *       e values:  y = o / (||o||_2 / sqrt(e)) (.) u,  and its gradients.
  *
  * Layout: q,k [B,H,N,d], v,o,dO [B,H,N,e], states [B,H,d,e] with
  * kv[i][j] = sum_s lambda^(t-s) k_s[i] v_s[j]; everything row-major contiguous.
@@ -32,7 +35,11 @@
  *     dQ_i += dA_ij K_j (the printed right-hand sides do not type-check), and
  *     O is not an input of the backward pass;
  *   - the state starts at zero unless kv_in is given; kv_out is the state after
- *     the last token with no extra decay.
+ *     the last token with no extra decay;
+ *   - SimpleRMSNorm is applied to each head's e output values of a token (the
+ *     model-parallel form of Eq. 3 normalises each rank's heads on their own);
+ *     Eq. 8 has no epsilon, so a row with ||o||_2 = 0 is given y = 0 and zero
+ *     gradients.
  *
  * Every routine is pinned by tests that do not call it twice: closed forms,
  * a hand-worked example, numpy prefix sums for lambda = 1, brute force on tiny
@@ -367,4 +374,49 @@ int orc_fwd_origin(const float* q, const float* k, const float* v, const double*
     free(kv);
   }
   return failed ? ORC_ERR : ORC_OK;
+}
+
+/*
+ * Eq. 3 with Eq. 8: y = SRMSNorm(o) (.) u per row of e values, SRMSNorm(x) = x / (||x||_2 / sqrt(e)).
+ * o [rows, e] fp64 (the attention output), u [rows, e] (exact input values), y [rows, e] fp64,
+ * rstd [rows] = sqrt(e) / ||o||_2 (0 for a zero row), or NULL.
+ */
+int orc_norm_gate_fwd(const double* o, const float* u, long rows, int e, double* y, double* rstd) {
+  if (!o || !u || !y || rows < 0 || e < 1) return ORC_ERR;
+#pragma omp parallel for schedule(static)
+  for (long r = 0; r < rows; ++r) {
+    const double* orow = o + r * e;
+    double ss = 0.0;
+    for (int j = 0; j < e; ++j) ss += orow[j] * orow[j];
+    const double s = ss > 0.0 ? sqrt((double)e) / sqrt(ss) : 0.0;
+    if (rstd) rstd[r] = s;
+    for (int j = 0; j < e; ++j) y[r * e + j] = orow[j] * s * (double)u[r * e + j];
+  }
+  return ORC_OK;
+}
+
+/*
+ * Gradients of L = <y, dy> with respect to o and u.  With n = o s, s = sqrt(e) / ||o||_2 and g = dy (.) u:
+ *   du = dy (.) n,     do = s (g - n (n . g) / e)
+ * (the second from d(o / ||o||) = (I - o o^T / ||o||^2) / ||o||; it is orthogonal to o because the norm
+ * removes the scale of o).
+ */
+int orc_norm_gate_bwd(const double* o, const float* u, const float* dy, long rows, int e, double* d_o,
+                      double* d_u) {
+  if (!o || !u || !dy || !d_o || !d_u || rows < 0 || e < 1) return ORC_ERR;
+#pragma omp parallel for schedule(static)
+  for (long r = 0; r < rows; ++r) {
+    const double* orow = o + r * e;
+    double ss = 0.0;
+    for (int j = 0; j < e; ++j) ss += orow[j] * orow[j];
+    const double s = ss > 0.0 ? sqrt((double)e) / sqrt(ss) : 0.0;
+    double ng = 0.0;
+    for (int j = 0; j < e; ++j) ng += (orow[j] * s) * ((double)dy[r * e + j] * (double)u[r * e + j]);
+    for (int j = 0; j < e; ++j) {
+      const double n = orow[j] * s, g = (double)dy[r * e + j] * (double)u[r * e + j];
+      d_u[r * e + j] = (double)dy[r * e + j] * n;
+      d_o[r * e + j] = s * (g - n * ng / (double)e);
+    }
+  }
+  return ORC_OK;
 }

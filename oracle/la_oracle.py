@@ -50,8 +50,10 @@ def _load():
         lib.orc_rows.argtypes = [I, fp, fp, fp, fp, dp, I, I, I, I, I, I, ip, ip, dp]
         lib.orc_decode_step.argtypes = [fp, fp, fp, dp, dp, I, I, I, I, dp]
         lib.orc_fwd_origin.argtypes = [fp, fp, fp, dp, I, I, I, I, I, dp]
+        lib.orc_norm_gate_fwd.argtypes = [dp, fp, ctypes.c_long, I, dp, dp]
+        lib.orc_norm_gate_bwd.argtypes = [dp, fp, fp, ctypes.c_long, I, dp, dp]
         for name in ("orc_fwd_rec", "orc_bwd_rec", "orc_fwd_quad", "orc_bwd_quad", "orc_rows",
-                     "orc_decode_step", "orc_fwd_origin"):
+                     "orc_decode_step", "orc_fwd_origin", "orc_norm_gate_fwd", "orc_norm_gate_bwd"):
             getattr(lib, name).restype = I
         _lib = lib
     return _lib
@@ -197,3 +199,32 @@ def fwd_origin(q, k, v, lam):
     _check(_load().orc_fwd_origin(_p(q, F), _p(k, F), _p(v, F), _p(lam, D), B, H, N, d, e, _p(o, D)),
            "orc_fwd_origin")
     return o
+
+
+def norm_gate_fwd(o, u, want_rstd: bool = False):
+    """y = SRMSNorm(o) (.) u per row of the last axis (Eq. 3 with Eq. 8). o fp64 array, u any; returns fp64."""
+    o = np.ascontiguousarray(np.asarray(o, np.float64))
+    u = _f32(u)
+    assert o.shape == u.shape
+    e = o.shape[-1]
+    rows = o.size // e
+    y = np.empty_like(o)
+    rstd = np.empty(o.shape[:-1], np.float64) if want_rstd else None
+    D, F = ctypes.c_double, ctypes.c_float
+    _check(_load().orc_norm_gate_fwd(_p(o, D), _p(u, F), ctypes.c_long(rows), e, _p(y, D), _p(rstd, D)),
+           "orc_norm_gate_fwd")
+    return (y, rstd) if want_rstd else y
+
+
+def norm_gate_bwd(o, u, dy):
+    """Gradients of <y, dy> with respect to o and u; returns (do, du) in fp64."""
+    o = np.ascontiguousarray(np.asarray(o, np.float64))
+    u, dy = _f32(u), _f32(dy)
+    assert o.shape == u.shape == dy.shape
+    e = o.shape[-1]
+    rows = o.size // e
+    d_o, d_u = np.empty_like(o), np.empty_like(o)
+    D, F = ctypes.c_double, ctypes.c_float
+    _check(_load().orc_norm_gate_bwd(_p(o, D), _p(u, F), _p(dy, F), ctypes.c_long(rows), e, _p(d_o, D), _p(d_u, D)),
+           "orc_norm_gate_bwd")
+    return d_o, d_u

@@ -387,3 +387,45 @@ def test_generator_is_seeded_and_bf16_exact():
     q = inputs.make_qkvdo(1, 4, 4096, 64, 64, seed=0, dtype=torch.float32)[0]
     assert abs(q.mean().item() - 0.20662) < 2e-3
     assert abs((q * q).mean().item() - 0.35578) < 4e-3
+
+
+# --- SimpleRMSNorm followed by the gate (Eq. 3 with Eq. 8) ---------------------------------
+def test_norm_gate_hand_worked_example():
+    g = json.load(open(os.path.join(HERE, "golden", "norm_gate_example.json")))
+    o = np.array(g["o"]).reshape(1, 2)
+    u = np.array(g["u"], np.float32).reshape(1, 2)
+    dy = np.array(g["dy"], np.float32).reshape(1, 2)
+    y, rstd = orc.norm_gate_fwd(o, u, want_rstd=True)
+    assert np.allclose(y.ravel(), g["y"], rtol=1e-15) and abs(rstd[0] - g["rstd"]) < 1e-16
+    d_o, d_u = orc.norm_gate_bwd(o, u, dy)
+    assert np.allclose(d_o.ravel(), g["do"], rtol=1e-14) and np.allclose(d_u.ravel(), g["du"], rtol=1e-15)
+
+
+def test_norm_gate_invariants_and_finite_differences():
+    rng = np.random.default_rng(7)
+    rows, e = 6, 5
+    o = rng.standard_normal((rows, e)) * np.array([1e-3, 1, 10, 1e3, 1, 1])[:, None]
+    u = rng.standard_normal((rows, e)).astype(np.float32)
+    dy = rng.standard_normal((rows, e)).astype(np.float32)
+    y = orc.norm_gate_fwd(o, u)
+    # the normalised row has root-mean-square 1, whatever the scale of o
+    assert np.allclose(np.sqrt(np.mean((y / u) ** 2, axis=1)), 1.0, rtol=1e-13)
+    # scale invariance of the norm: y(a o) = y(o); do(a o) = do(o) / a; do is orthogonal to o
+    d_o, d_u = orc.norm_gate_bwd(o, u, dy)
+    assert np.allclose(orc.norm_gate_fwd(7.5 * o, u), y, rtol=1e-13)
+    assert np.allclose(orc.norm_gate_bwd(7.5 * o, u, dy)[0], d_o / 7.5, rtol=1e-12)
+    assert np.all(np.abs(np.sum(o * d_o, axis=1)) <= 1e-12 * np.linalg.norm(o, axis=1) * np.linalg.norm(d_o, axis=1))
+    # central differences of L = <y, dy> in o and in u
+    L = lambda oo, uu: float(np.sum(orc.norm_gate_fwd(oo, uu) * dy))
+    for (r, j) in [(0, 1), (2, 4), (3, 0), (5, 2)]:
+        h = 1e-6 * max(1.0, abs(o[r, j]))
+        op, om = o.copy(), o.copy()
+        op[r, j] += h
+        om[r, j] -= h
+        fd = (L(op, u) - L(om, u)) / (2 * h)
+        assert abs(fd - d_o[r, j]) <= 1e-6 * max(abs(fd), np.abs(d_o[r]).max())
+        # L is linear in u: the derivative is dy * n, exactly the forward value divided by u
+        assert abs(d_u[r, j] - dy[r, j] * y[r, j] / u[r, j]) <= 1e-12 * abs(d_u[r, j]) + 1e-300
+    # a zero row is given y = 0 and zero gradients (Eq. 8 has no epsilon)
+    z = np.zeros((1, e))
+    assert np.all(orc.norm_gate_fwd(z, u[:1]) == 0) and np.all(orc.norm_gate_bwd(z, u[:1], dy[:1])[0] == 0)
