@@ -329,6 +329,49 @@ def run_ours(args):
         barrier()
         split_ms[nm] = max_over_ranks(s0.elapsed_time(s1) / nrep)
 
+    # ---- the token mixer's output stage fused into the forward walk (y = SRMSNorm(o) (.) u), same shape ----
+    gated = None
+    if train_steps:
+        gen_u = torch.Generator(dev)
+        gen_u.manual_seed(77 + rank)
+        ug = torch.randn((w.B, w.H, w.N, w.e), generator=gen_u, device=dev).to(torch.bfloat16)
+        yg = torch.empty_like(o)
+        dyg = torch.randn((w.B, w.H, w.N, w.e), generator=gen_u, device=dev).to(torch.bfloat16)
+        dog = torch.empty((w.B, w.H, w.N, w.e), dtype=torch.bfloat16, device=dev)
+
+        def time_loop(fn, n=10):
+            fn()
+            barrier()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            l0 = la.launch_count()
+            a0.record(stream)
+            for _ in range(n):
+                fn()
+            a1.record(stream)
+            barrier()
+            la.device_status()
+            return max_over_ranks(a0.elapsed_time(a1) / n), (la.launch_count() - l0) / n
+
+        fused_ms, fused_l = time_loop(lambda: la.la_fwd_gated(shape, q, k, v, ug, lam, yg, None, None, None, None, ws_f, stream))
+        train_ms, train_l = time_loop(lambda: la.la_fwd_gated(shape, q, k, v, ug, lam, yg, o, None, None, None, ws_f, stream))
+
+        def unfused():
+            la.la_fwd(shape, q, k, v, lam, o, None, None, ws_f, stream)
+            la.la_gate_fwd(shape, o, ug, yg, None, stream)
+
+        unfused_ms, unfused_l = time_loop(unfused)
+        gbwd_ms, _ = time_loop(lambda: la.la_gate_bwd(shape, o, ug, dyg, dog, dv, stream))
+        eb = 4 if out_dtype == torch.float32 else 2
+        gated = {"what": "la_fwd_gated at the same shape: y = SRMSNorm(o) (.) u as the forward walk's epilogue (Eq. 3, Eq. 8)",
+                 "fused_ms": fused_ms, "fused_launches": fused_l,
+                 "fused_bytes_per_token_head": 2 * 4 * w.d + eb * w.d,      # read q,k,v,u ; write y (o never written)
+                 "fused_also_writing_o_ms": train_ms,
+                 "unfused_ms": unfused_ms, "unfused_launches": unfused_l,
+                 "unfused_bytes_per_token_head": 2 * 4 * w.d + 3 * eb * w.d,  # + write o, read o back
+                 "gate_bwd_ms": gbwd_ms,
+                 "gate_bwd_gbs": th * (eb * w.d + 3 * 2 * w.d + eb * w.d) / (gbwd_ms * 1e-3) / 1e9}
+        del ug, yg, dyg, dog
+
     # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
     dw = inputs.WORKLOADS["decode"]
     gen = torch.Generator(dev)
@@ -487,7 +530,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / prof_steps for kname, (ms, _) in prof.items()},
             "kernel_launches_per_step": {kname: c / prof_steps for kname, (_, c) in prof.items()},
-            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"),
+            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated,
             "roofline": {"scope": "ONE kernel, the dominant one; the whole-step figure the target is stated on is step_roofline",
                          "kernel": "full-width block walk (tc_walk_full_kernel), single-job launches (O and dQ)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -119,6 +119,43 @@ la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void
                  void* workspace, size_t workspace_bytes, void* stream /* cudaStream_t */);
 
 /*
+ * Forward pass with the rest of the token mixer's output stage fused in (Eq. 3 "Gated Linear Attention" with
+ * Eq. 8 "SimpleRMSNorm"): per batch, head and token, with o the e attention outputs of la_fwd,
+ *   y = o / (||o||_2 / sqrt(e)) (.) u
+ * (each head's e values are normalised on their own, as in the model-parallel form of Eq. 3; Eq. 8 has no
+ * epsilon: a row with ||o||_2 = 0 gives y = 0).
+ *   u     [B,H,N,e] gate, in_dtype;
+ *   y     [B,H,N,e] out_dtype;
+ *   o     [B,H,N,e] out_dtype, the attention output itself, or NULL if it is not wanted (inference); the
+ *         backward of this stage (la_gate_bwd) needs it;
+ *   rstd  [B,H,N] fp32, sqrt(e) / ||o||_2 per row, or NULL.
+ * Everything else as for la_fwd.  At d = e = 128 on the tensor-core path, with y (and o) aligned to 32 bytes, the
+ * epilogue runs inside the walk kernel and o is never written unless asked for; otherwise the attention output is
+ * written (to o, or to y if o is NULL) and a row kernel turns it into y.
+ */
+la_status la_fwd_gated(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
+                       const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same output stage on its own (Eq. 3 with Eq. 8), for an attention output that already sits in memory:
+ *   y = o / (||o||_2 / sqrt(e)) (.) u;  o, y [B,H,N,e] out_dtype (they may be the same buffer), u in_dtype,
+ *   rstd [B,H,N] fp32 or NULL.  One bandwidth-bound row kernel; this is what la_fwd_gated runs behind the walk
+ *   where it cannot fuse.  shape->d is ignored.
+ */
+la_status la_gate_fwd(const la_shape* shape, const void* o, const void* u, void* y, float* rstd, void* stream);
+
+/*
+ * Backward of that output stage (the chain rule through Eq. 3 / Eq. 8): from d_y = dL/dy
+ *   d_u = d_y (.) n,      d_o = s (g - n (n . g) / e),      n = o s,  s = sqrt(e) / ||o||_2,  g = d_y (.) u.
+ *   o [B,H,N,e] out_dtype (as written by la_fwd_gated); u, d_y [B,H,N,e] in_dtype;
+ *   d_o [B,H,N,e] in_dtype (it is what la_bwd takes as d_o); d_u [B,H,N,e] out_dtype.
+ * One bandwidth-bound row kernel; needs no workspace.  shape->d is ignored.
+ */
+la_status la_gate_bwd(const la_shape* shape, const void* o, const void* u, const void* d_y, void* d_o, void* d_u,
+                      void* stream);
+
+/*
  * Backward pass (Algorithm 4 defines the result): gradients of
  * L = <O, dO> + <kv_out, grad_kv_out> with respect to q, k, v (and kv_in).
  *   d_o          [B,H,N,e] in in_dtype;
@@ -260,7 +297,8 @@ unsigned long long la_launch_count(void);
 #define LA_KERNEL_WALK 2    /* block walk producing o/dq/dk/dv */
 #define LA_KERNEL_DECODE 3  /* recurrent decode step           */
 #define LA_KERNEL_WALK_PAIR 4 /* the dV and dK walks of the backward pass in one launch */
-#define LA_NUM_KERNEL_KINDS 5
+#define LA_KERNEL_GATE 5      /* stand-alone SRMSNorm-and-gate kernels (la_fwd_gated fallback, la_gate_bwd) */
+#define LA_NUM_KERNEL_KINDS 6
 void la_profile_enable(int on);
 la_status la_profile_collect(double* ms, unsigned long long* launches);
 

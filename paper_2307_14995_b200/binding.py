@@ -25,9 +25,9 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
            "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
-           "la_selftest_bounded_wait")
+           "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
-KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair")
+KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate")
 
 
 class LaShape(ctypes.Structure):
@@ -62,6 +62,12 @@ def load():
         lib.la_segment_length.restype = I
         lib.la_fwd.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp, vp, sz, vp]
         lib.la_fwd.restype = I
+        lib.la_fwd_gated.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.la_fwd_gated.restype = I
+        lib.la_gate_fwd.argtypes = [sp, vp, vp, vp, vp, vp]
+        lib.la_gate_fwd.restype = I
+        lib.la_gate_bwd.argtypes = [sp, vp, vp, vp, vp, vp, vp]
+        lib.la_gate_bwd.restype = I
         lib.la_fwd_noalloc.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp, vp]
         lib.la_fwd_noalloc.restype = I
         lib.la_bwd.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -183,6 +189,28 @@ def la_fwd(shape: LaShape, q, k, v, lam, o, kv_in=None, kv_out=None, workspace=N
                        _ptr(kv_out), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_fwd")
+
+
+def la_fwd_gated(shape: LaShape, q, k, v, u, lam, y, o=None, rstd=None, kv_in=None, kv_out=None, workspace=None,
+                 stream=None):
+    """la_fwd with y = SRMSNorm(o) (.) u as its output stage; o and rstd are optional outputs."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_fwd_gated(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(u), _lam(lam), _ptr(y), _ptr(o),
+                             _ptr(rstd), _ptr(kv_in), _ptr(kv_out), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_fwd_gated")
+
+
+def la_gate_fwd(shape: LaShape, o, u, y, rstd=None, stream=None):
+    rc = load().la_gate_fwd(ctypes.byref(shape), _ptr(o), _ptr(u), _ptr(y), _ptr(rstd), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_gate_fwd")
+
+
+def la_gate_bwd(shape: LaShape, o, u, dy, d_o, d_u, stream=None):
+    rc = load().la_gate_bwd(ctypes.byref(shape), _ptr(o), _ptr(u), _ptr(dy), _ptr(d_o), _ptr(d_u), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_gate_bwd")
 
 
 def la_fwd_noalloc(shape: LaShape, q, k, v, lam, o, kv_in=None, kv_out=None, stream=None):

@@ -212,6 +212,10 @@ cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, co
   return launch_simt_walk(args, tab, s->d, s->e, (int)s->in_dtype, (int)s->out_dtype, st);
 }
 
+la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
+                   const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
 }  // namespace
 }  // namespace la
 
@@ -240,11 +244,54 @@ int la_segment_length(const la_shape* shape) {
 la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void* v,
                  const float* lambda_host, void* o, const float* kv_in, float* kv_out,
                  void* workspace, size_t workspace_bytes, void* stream) {
+  return fwd_impl(shape, q, k, v, nullptr, lambda_host, nullptr, o, nullptr, kv_in, kv_out, workspace, workspace_bytes,
+                  stream);
+}
+
+la_status la_fwd_gated(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
+                       const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+  if (!u || !y) return LA_ERR_INVALID_ARG;
+  return fwd_impl(shape, q, k, v, u, lambda_host, y, o, rstd, kv_in, kv_out, workspace, workspace_bytes, stream);
+}
+
+la_status la_gate_fwd(const la_shape* shape, const void* o, const void* u, void* y, float* rstd, void* stream) {
   la_status st = check_shape(shape, true);
   if (st != LA_OK) return st;
-  if (!q || !k || !v || !o) return LA_ERR_INVALID_ARG;
+  if (!o || !u || !y) return LA_ERR_INVALID_ARG;
+  if (!aligned16(o) || !aligned16(u) || !aligned16(y) || !aligned16(rstd)) return LA_ERR_INVALID_ARG;
+  if ((st = check_device()) != LA_OK) return st;
+  LA_TRY_CUDA(launch_norm_gate_fwd(o, u, y, rstd, (long)shape->B * shape->H * shape->N, shape->e, (int)shape->in_dtype,
+                                   (int)shape->out_dtype, static_cast<cudaStream_t>(stream)));
+  return LA_OK;
+}
+
+la_status la_gate_bwd(const la_shape* shape, const void* o, const void* u, const void* d_y, void* d_o, void* d_u,
+                      void* stream) {
+  la_status st = check_shape(shape, true);
+  if (st != LA_OK) return st;
+  if (!o || !u || !d_y || !d_o || !d_u) return LA_ERR_INVALID_ARG;
+  if (!aligned16(o) || !aligned16(u) || !aligned16(d_y) || !aligned16(d_o) || !aligned16(d_u)) return LA_ERR_INVALID_ARG;
+  if ((st = check_device()) != LA_OK) return st;
+  LA_TRY_CUDA(launch_norm_gate_bwd(o, u, d_y, d_o, d_u, (long)shape->B * shape->H * shape->N, shape->e,
+                                   (int)shape->in_dtype, (int)shape->out_dtype, static_cast<cudaStream_t>(stream)));
+  return LA_OK;
+}
+
+}  // extern "C"
+
+namespace la {
+namespace {
+// la_fwd and la_fwd_gated: u == NULL is the plain forward pass (o required); with u the rows leave as
+// y = SRMSNorm(o) (.) u, fused into the walk where the kernel can, else by a row kernel behind it.
+la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
+                   const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
+                   void* workspace, size_t workspace_bytes, void* stream) {
+  la_status st = check_shape(shape, true);
+  if (st != LA_OK) return st;
+  if (!q || !k || !v || (!u && !o)) return LA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(kv_in) ||
-      !aligned16(kv_out))
+      !aligned16(kv_out) || !aligned16(u) || !aligned16(y) || !aligned16(rstd))
     return LA_ERR_INVALID_ARG;
   DecayTable tab;
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
@@ -263,9 +310,29 @@ la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void
     LA_TRY_CUDA(run_scan(shape, p, tab, buf, nullptr, kv_in, false, 0, cs));
     entry = buf;
   }
-  LA_TRY_CUDA(run_walk(shape, p, tab, q, k, v, o, entry, kv_out, 0, cs));
+  if (!u) {
+    LA_TRY_CUDA(run_walk(shape, p, tab, q, k, v, o, entry, kv_out, 0, cs));
+    return LA_OK;
+  }
+  OpArgs wa = walk_args(shape, p, q, k, v, o, entry, kv_out, 0);
+  wa.u = u;
+  wa.y = y;
+  wa.rstd = rstd;
+  if (p.tensor && tc_can_fuse_gate(wa, shape->d)) {
+    LA_TRY_CUDA(launch_tc_walk(wa, tab, shape->d, (int)shape->out_dtype, p.precision, cs));
+    return LA_OK;
+  }
+  // not fused: the attention output goes to o (or, if it is not wanted, to y itself) and a row kernel turns it into y
+  void* att = o ? o : y;
+  LA_TRY_CUDA(run_walk(shape, p, tab, q, k, v, att, entry, kv_out, 0, cs));
+  LA_TRY_CUDA(launch_norm_gate_fwd(att, u, y, rstd, (long)p.BH * shape->N, shape->e, (int)shape->in_dtype,
+                                   (int)shape->out_dtype, cs));
   return LA_OK;
 }
+}  // namespace
+}  // namespace la
+
+extern "C" {
 
 la_status la_bwd(const la_shape* shape, const void* q, const void* k, const void* v,
                  const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,

@@ -48,6 +48,11 @@ struct OpArgs {
   int BH, H, N;
   int seg_len, nseg;  // seg_len is a multiple of 128
   int reverse;        // 0 forward, 1 reverse
+  // Optional epilogue of the forward walk (Eq. 3 with Eq. 8): y = SRMSNorm(out) (.) u per row.  With u set, y is
+  // written, `out` becomes optional (NULL = the attention output itself is not wanted) and rstd [BH, N] optional.
+  const void* u;      // [BH, N, Ec] gate, input dtype
+  void* y;            // [BH, N, Ec] output dtype
+  float* rstd;        // [BH, N] sqrt(Ec) / ||out row||_2, or NULL
 };
 
 struct ScanArgs {
@@ -73,10 +78,20 @@ cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv
                           int H, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
                           cudaStream_t stream);
 
+// SimpleRMSNorm followed by the gate as stand-alone row kernels (la_gate.cu): y = SRMSNorm(o) (.) u (o and y may be
+// the same buffer), and the gradients of <y, dy> with respect to o (written in the input dtype) and u.
+cudaError_t launch_norm_gate_fwd(const void* o, const void* u, void* y, float* rstd, long rows, int e, int in_dt,
+                                 int out_dt, cudaStream_t stream);
+cudaError_t launch_norm_gate_bwd(const void* o, const void* u, const void* dy, void* d_o, void* d_u, long rows, int e,
+                                 int in_dt, int out_dt, cudaStream_t stream);
+
 // Tensor-core (tcgen05) kernels: bf16 inputs, Da = Ec = D with D = 64 or 128.
 bool tc_supported();
 cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int out_dt, int precision,
                            cudaStream_t stream);
+// Whether launch_tc_walk can fuse the epilogue described by args.u / args.y into the walk (d = 128, y and out
+// aligned to 32 bytes); otherwise the caller runs the walk and then launch_norm_gate_fwd.
+bool tc_can_fuse_gate(const OpArgs& args, int D);
 // Two walks of the same direction over the same tokens (same N, BH, segments) in one launch; the thread blocks of
 // the two are interleaved so that tiles both read come from HBM once.
 // Whether the d = 128 walk normally runs as one full-width thread block per (head, segment) rather than two
@@ -106,7 +121,7 @@ struct KernelTimer {
   cudaEvent_t start_;
   bool active_;
 };
-enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_WALK_PAIR = 4, K_NUM = 5 };
+enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_WALK_PAIR = 4, K_GATE = 5, K_NUM = 6 };
 
 // ---- small device helpers --------------------------------------------------
 __device__ __forceinline__ float decay_pow(float s2, float n) {

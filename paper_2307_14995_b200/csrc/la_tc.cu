@@ -104,6 +104,10 @@ struct TcJob {
   void* out;
   const float* entry;
   float* final_out;
+  // gate epilogue of the forward walk (full-width kernel only): y = SRMSNorm(out) (.) u
+  const void* u;
+  void* y;
+  float* rstd;
 };
 
 struct TcMaps {
@@ -849,7 +853,8 @@ cudaError_t launch_t(const TcMaps& m0, const TcMaps& m1, const TcArgs& ta, const
 
 bool make_maps(TcMaps* m, const OpArgs& args, int D, bool f32) {
   return make_map(&m->a, args.a, args.N, args.BH, D) && make_map(&m->b, args.b, args.N, args.BH, D) &&
-         make_map(&m->c, args.c, args.N, args.BH, D) && make_map(&m->out, args.out, args.N, args.BH, D, f32);
+         make_map(&m->c, args.c, args.N, args.BH, D) &&
+         make_map(&m->out, args.out ? args.out : args.y, args.N, args.BH, D, f32);  // (gated walk without `out`: y)
 }
 
 // One walk (second == nullptr) or two walks of the same direction over the same tokens in one launch.
@@ -865,26 +870,32 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
     m1 = m0;
   }
   TcArgs ta{};
-  ta.job[0] = TcJob{args.c, args.out, args.entry, args.final_out};
-  ta.job[1] = second ? TcJob{second->c, second->out, second->entry, second->final_out} : ta.job[0];
+  ta.job[0] = TcJob{args.c, args.out, args.entry, args.final_out, args.u, args.y, args.rstd};
+  ta.job[1] = second ? TcJob{second->c, second->out, second->entry, second->final_out, nullptr, nullptr, nullptr} : ta.job[0];
   ta.local_out = nullptr;
   ta.njobs = second ? 2 : 1;
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
+  if (args.u) {
+    // forward walk with the gate epilogue: only the full-width kernel has it (the caller asks tc_can_fuse_gate first)
+    if (D != 128 || second || args.reverse || !tc_can_fuse_gate(args, D)) return cudaErrorInvalidValue;
+    return f32 ? launch_full_t<false, float, 1, true>(m0, m1, ta, tab, stream)
+               : launch_full_t<false, __nv_bfloat16, 1, true>(m0, m1, ta, tab, stream);
+  }
   if (D == 128 && !(reinterpret_cast<uintptr_t>(args.out) & 31u) &&
       !(second && (reinterpret_cast<uintptr_t>(second->out) & 31u))) {
     // full-width kernel: one thread block per (head, segment).  Its 32-byte output stores need that alignment;
     // an output that is only 16-byte aligned (the contract's minimum) takes the half-width kernels below.
     if (second) {
       if (!args.reverse) return cudaErrorInvalidValue;
-      return f32 ? launch_full_t<true, float, 2>(m0, m1, ta, tab, stream)
-                 : launch_full_t<true, __nv_bfloat16, 2>(m0, m1, ta, tab, stream);
+      return f32 ? launch_full_t<true, float, 2, false>(m0, m1, ta, tab, stream)
+                 : launch_full_t<true, __nv_bfloat16, 2, false>(m0, m1, ta, tab, stream);
     }
     if (args.reverse)
-      return f32 ? launch_full_t<true, float, 1>(m0, m1, ta, tab, stream)
-                 : launch_full_t<true, __nv_bfloat16, 1>(m0, m1, ta, tab, stream);
-    return f32 ? launch_full_t<false, float, 1>(m0, m1, ta, tab, stream)
-               : launch_full_t<false, __nv_bfloat16, 1>(m0, m1, ta, tab, stream);
+      return f32 ? launch_full_t<true, float, 1, false>(m0, m1, ta, tab, stream)
+                 : launch_full_t<true, __nv_bfloat16, 1, false>(m0, m1, ta, tab, stream);
+    return f32 ? launch_full_t<false, float, 1, false>(m0, m1, ta, tab, stream)
+               : launch_full_t<false, __nv_bfloat16, 1, false>(m0, m1, ta, tab, stream);
   }
   if (second) {  // only the reverse direction is ever paired
     if (!args.reverse) return cudaErrorInvalidValue;
@@ -907,7 +918,7 @@ cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int prec
   m.a = m.b;
   m.out = m.c;
   TcArgs ta{};
-  ta.job[0] = TcJob{args.c, nullptr, nullptr, nullptr};
+  ta.job[0] = TcJob{args.c, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   ta.job[1] = ta.job[0];
   ta.local_out = args.local_out;
   ta.njobs = 1;
@@ -928,6 +939,13 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int
 }
 
 bool tc_full_width() { return true; }
+
+bool tc_can_fuse_gate(const OpArgs& args, int D) {
+  if (D != 128 || !args.u || !args.y) return false;
+  if (reinterpret_cast<uintptr_t>(args.y) & 31u) return false;
+  if (args.out && (reinterpret_cast<uintptr_t>(args.out) & 31u)) return false;
+  return true;
+}
 
 cudaError_t launch_tc_walk_pair(const OpArgs& first, const OpArgs& second, const DecayTable& tab, int D, int out_dt,
                                 int precision, cudaStream_t stream) {

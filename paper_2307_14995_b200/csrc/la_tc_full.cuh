@@ -69,7 +69,9 @@ __device__ __forceinline__ void reg_inc() {
 // NJOBS = 2: two walks of the same direction over the same tokens in one launch (the dV and dK walks of the backward
 // pass, which between them read Q, K, V and dO); the thread blocks of the two jobs alternate, so that the two
 // readers of a tile run side by side and the tile comes from HBM once.
-template <bool REV, typename TOut, int NJOBS>
+// GATED (forward, single job): the epilogue y = SRMSNorm(out) (.) u of Eq. 3 with Eq. 8 is applied to the rows
+// before they leave (job.u, job.y; job.out and job.rstd optional).
+template <bool REV, typename TOut, int NJOBS, bool GATED>
 __global__ void __launch_bounds__(F_THREADS, 1)
 tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps maps1, const TcArgs args,
                     const DecayTable tab) {
@@ -381,7 +383,9 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const bool b0 = (lane & 1) != 0, b1 = (lane & 2) != 0;
     const int g = lane & 3;
-    constexpr int COLS = 128 / (int)sizeof(TOut);  // columns per 128-byte piece: 32 fp32 or 64 bf16
+    // columns per 128-byte piece: 32 fp32 or 64 bf16; with the gate the rows stay fp32 until they are stored
+    constexpr bool F32ROWS = GATED || sizeof(TOut) == 4;
+    constexpr int COLS = F32ROWS ? 32 : 64;
     constexpr int NPIECE = 128 / COLS;             // 4 or 2
     const int ohalf = (warp >= 28) ? 1 : 0;        // warps 8..11 take the first half of the pieces, 28..31 the second
     for (int it = 0; it < nblk; ++it) {
@@ -395,6 +399,28 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
       // O_READY: every product up to M4 of this block is done
       TC_WAIT_WARP(F_O_READY, it & 1, 25);
       tc_fence_after_sync();
+      float srow[4] = {0.f, 0.f, 0.f, 0.f};  // gate: sqrt(128) / ||row|| of the rows of lanes ^ 0..3
+      if (GATED) {
+        // first pass over the whole row (both halves of the columns: each warp of a pair does this for itself, which
+        // costs tensor-memory reads but no exchange between warps): sum of squares of out = O_intra + f O_inter
+        float ss = 0.f;
+#pragma unroll
+        for (int sub = 0; sub < 8; ++sub) {
+          uint32_t oi[16], oe[16];
+          tmem_ld_x16(lane_addr + FCOL_OI + sub * 16, oi);
+          tmem_ld_x16(lane_addr + FCOL_OE + sub * 16, oe);
+          tmem_ld_wait();
+#pragma unroll
+          for (int x = 0; x < 16; ++x) {
+            const float v = fmaf(f, __uint_as_float(oe[x]), __uint_as_float(oi[x]));
+            ss = fmaf(v, v, ss);
+          }
+        }
+        const float s = ss > 0.f ? rsqrtf(ss * (1.f / 128.f)) : 0.f;
+        if (job.rstd && ohalf == 0 && r < Cr) job.rstd[(size_t)bh * args.N + t0 + r] = s;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) srow[k] = __shfl_xor_sync(0xffffffffu, s, k);
+      }
 #pragma unroll
       for (int pcl = 0; pcl < NPIECE / 2; ++pcl) {
         const int pc = ohalf * (NPIECE / 2) + pcl;
@@ -410,7 +436,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
             tc_fence_before_sync();
             WARP_ARRIVE(F_O_FREE);  // both accumulators are in registers: M2 and M4 of the next block may overwrite them
           }
-          if (sizeof(TOut) == 4) {
+          if (F32ROWS) {
 #pragma unroll
             for (int x = 0; x < 16; ++x)
               w[sub * 16 + x] = __float_as_uint(fmaf(f, __uint_as_float(oe[x]), __uint_as_float(oi[x])));
@@ -448,8 +474,39 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int row_in_quad = g ^ k;  // slot k holds the row of lane ^ k
-          if ((r & ~3) + row_in_quad < Cr)
+          if ((r & ~3) + row_in_quad >= Cr) continue;
+          if (!GATED) {
             st_global_v8(quad_base + (size_t)row_in_quad * (128 * sizeof(TOut)) + pc * 128, &w[8 * k]);
+          } else {
+            // slot k: columns pc * 32 + 8 g .. + 8 of that row, still fp32
+            const size_t elem = ((size_t)bh * args.N + t0 + (r & ~3) + row_in_quad) * 128 + pc * 32 + g * 8;
+            const uint4 uraw = __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.u) + elem));
+            const uint32_t uw[4] = {uraw.x, uraw.y, uraw.z, uraw.w};
+            uint32_t yv[8];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              const float2 ug = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&uw[x]));
+              yv[2 * x] = __float_as_uint(__uint_as_float(w[8 * k + 2 * x]) * srow[k] * ug.x);
+              yv[2 * x + 1] = __float_as_uint(__uint_as_float(w[8 * k + 2 * x + 1]) * srow[k] * ug.y);
+            }
+            if (sizeof(TOut) == 4) {
+              st_global_v8(static_cast<float*>(job.y) + elem, yv);
+              if (job.out) st_global_v8(static_cast<float*>(job.out) + elem, &w[8 * k]);
+            } else {
+              uint4 yp, op;
+              uint32_t* ypw = reinterpret_cast<uint32_t*>(&yp);
+              uint32_t* opw = reinterpret_cast<uint32_t*>(&op);
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(yv[2 * x]), __uint_as_float(yv[2 * x + 1]));
+                const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(w[8 * k + 2 * x]), __uint_as_float(w[8 * k + 2 * x + 1]));
+                ypw[x] = *reinterpret_cast<const uint32_t*>(&a);
+                opw[x] = *reinterpret_cast<const uint32_t*>(&b);
+              }
+              *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(job.y) + elem) = yp;
+              if (job.out) *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(job.out) + elem) = op;
+            }
+          }
         }
       }
     }
@@ -474,10 +531,10 @@ teardown:
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-template <bool REV, typename TOut, int NJOBS>
+template <bool REV, typename TOut, int NJOBS, bool GATED>
 cudaError_t launch_full_t(const TcMaps& m0, const TcMaps& m1, const TcArgs& ta, const DecayTable& tab, cudaStream_t stream) {
   const size_t smem = sizeof(FSmem) + 1024;
-  auto kern = tc_walk_full_kernel<REV, TOut, NJOBS>;
+  auto kern = tc_walk_full_kernel<REV, TOut, NJOBS, GATED>;
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   KernelTimer timer(NJOBS == 2 ? K_WALK_PAIR : K_WALK, stream);
