@@ -290,6 +290,7 @@ def run_ours(args):
 
     th = w.token_heads
     F = flops_per_token_head(w.d)
+    ms_step = max(ms_step, 1e-9)  # (--only decode times no training step)
     value = world * th * F / (ms_step * 1e-3) / 1e12
     ob = 4 if out_dtype == torch.float32 else 2
     step_bytes = th * bytes_per_token_head(w.d, ob, "step")

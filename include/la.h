@@ -194,6 +194,18 @@ la_status la_decode_step(const la_shape* shape, const void* q, const void* k, co
                          const float* lambda_host, float* kv, void* o, void* stream);
 
 /*
+ * Several recurrent decode steps in one call (Algorithm 2 iterated over shape->N >= 1 consecutive tokens): for
+ * t = 0 .. N-1 in order,  kv <- lambda_h kv + k_t v_t^T,  o_t <- kv^T q_t.
+ *   q, k [B,H,N,d], v [B,H,N,e] in in_dtype; o [B,H,N,e] in out_dtype; kv [B,H,d,e] fp32, updated IN PLACE once.
+ * The state is read once, kept on chip over the N tokens and written once, so a handful of tokens decoded together
+ * (speculative decoding, a short chunk of a prompt) costs one pass over the state instead of N.  The tokens are
+ * processed one after the other; for long chunks la_fwd with kv_in / kv_out is the faster route.  Same result
+ * as N calls of la_decode_step, bit for bit.  Needs no workspace, keeps no host state.
+ */
+la_status la_decode_steps(const la_shape* shape, const void* q, const void* k, const void* v,
+                          const float* lambda_host, float* kv, void* o, void* stream);
+
+/*
  * Forward pass without caller-provided scratch (the paper has no counterpart; this is a
  * deployment convenience).  Same result as la_fwd, but the per-segment state scratch comes
  * from a fixed LA_NOALLOC_SCRATCH_BYTES array that is part of the library's device image,

@@ -25,7 +25,7 @@ LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
            "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
-           "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd")
+           "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd", "la_decode_steps")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate")
 
@@ -76,6 +76,8 @@ def load():
         lib.la_bwd_reuse.restype = I
         lib.la_decode_step.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_step.restype = I
+        lib.la_decode_steps.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
+        lib.la_decode_steps.restype = I
         lib.la_host_arena_bytes.argtypes = [sp]
         lib.la_host_arena_bytes.restype = sz
         lib.la_fwd_bwd_host.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, vp, vp, sz, vp]
@@ -246,6 +248,14 @@ def la_decode_step(shape: LaShape, q, k, v, lam, kv, o, stream=None):
                                _ptr(o), _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_decode_step")
+
+
+def la_decode_steps(shape: LaShape, q, k, v, lam, kv, o, stream=None):
+    """shape.N consecutive tokens per call: q, k [B,H,N,d], v, o [B,H,N,e]; kv updated in place once."""
+    rc = load().la_decode_steps(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(kv),
+                                _ptr(o), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_decode_steps")
 
 
 def host_arena_bytes(shape: LaShape) -> int:

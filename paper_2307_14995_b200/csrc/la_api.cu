@@ -215,6 +215,8 @@ cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, co
 la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
                    const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
                    void* workspace, size_t workspace_bytes, void* stream);
+la_status decode_impl(const la_shape* shape, int T, const void* q, const void* k, const void* v,
+                      const float* lambda_host, float* kv, void* o, void* stream);
 
 }  // namespace
 }  // namespace la
@@ -408,6 +410,21 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
 
 la_status la_decode_step(const la_shape* shape, const void* q, const void* k, const void* v,
                          const float* lambda_host, float* kv, void* o, void* stream) {
+  return decode_impl(shape, 1, q, k, v, lambda_host, kv, o, stream);
+}
+
+la_status la_decode_steps(const la_shape* shape, const void* q, const void* k, const void* v,
+                          const float* lambda_host, float* kv, void* o, void* stream) {
+  if (!shape || shape->N < 1) return LA_ERR_INVALID_ARG;
+  return decode_impl(shape, shape->N, q, k, v, lambda_host, kv, o, stream);
+}
+
+}  // extern "C"
+
+namespace la {
+namespace {
+la_status decode_impl(const la_shape* shape, int T, const void* q, const void* k, const void* v,
+                      const float* lambda_host, float* kv, void* o, void* stream) {
   la_status st = check_shape(shape, false);
   if (st != LA_OK) return st;
   if (!q || !k || !v || !kv || !o) return LA_ERR_INVALID_ARG;
@@ -416,11 +433,15 @@ la_status la_decode_step(const la_shape* shape, const void* q, const void* k, co
   DecayTable tab;
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
   if ((st = check_device()) != LA_OK) return st;
-  LA_TRY_CUDA(launch_decode(q, k, v, kv, o, shape->B * shape->H, shape->H, shape->d, shape->e,
+  LA_TRY_CUDA(launch_decode(q, k, v, kv, o, shape->B * shape->H, shape->H, T, shape->d, shape->e,
                             (int)shape->in_dtype, (int)shape->out_dtype, tab,
                             static_cast<cudaStream_t>(stream)));
   return LA_OK;
 }
+}  // namespace
+}  // namespace la
+
+extern "C" {
 
 static size_t round256(size_t n) { return (n + 255) / 256 * 256; }
 

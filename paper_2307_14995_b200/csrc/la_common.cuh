@@ -74,8 +74,9 @@ cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int D
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream);
 // dst[m] = transpose(src[m]) for `count` row-major Da x Ec fp32 matrices.
 cudaError_t launch_transpose_states(const float* src, float* dst, long count, int Da, int Ec, cudaStream_t stream);
+// T >= 1 consecutive tokens per (batch, head): q, k [BH, T, d], v, o [BH, T, e].
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv, void* o, int BH,
-                          int H, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
+                          int H, int T, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
                           cudaStream_t stream);
 
 // SimpleRMSNorm followed by the gate as stand-alone row kernels (la_gate.cu): y = SRMSNorm(o) (.) u (o and y may be

@@ -1,5 +1,8 @@
-// Recurrent decode step (one iteration of Algorithm 2) for all (batch, head) pairs:
-//   kv <- lambda kv + k v^T,   o <- kv^T q,   kv fp32 [BH, d, e] updated in place.
+// Recurrent decode (iterations of Algorithm 2) for all (batch, head) pairs:
+//   kv <- lambda kv + k v^T,   o <- kv^T q,   kv fp32 [BH, d, e] updated in place,
+// for T >= 1 consecutive tokens per launch (q, k [BH, T, d], v, o [BH, T, e]): the state is read once, kept in
+// registers over the T tokens and written once, so a few tokens decoded together (speculative or chunked
+// decoding) cost one pass over the state instead of T.
 //
 // The step moves 2*d*e*4 bytes of state per (b,h) against 5*d*e flops, so it is
 // bound by HBM bandwidth and runs on the plain fp32 ALUs.  One thread block owns
@@ -17,7 +20,7 @@ constexpr int THREADS = 256;
 template <typename TIn, typename TOut, int D, int E>
 __global__ void __launch_bounds__(THREADS)
 decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
-              float* __restrict__ kv, TOut* __restrict__ o, int H, const DecayTable tab) {
+              float* __restrict__ kv, TOut* __restrict__ o, int H, int T, const DecayTable tab) {
   constexpr int LPR = E / 4;              // lanes per state row (float4 each)
   constexpr int RPP = THREADS / LPR;      // rows per pass
   constexpr int PASSES = D / RPP;
@@ -40,81 +43,87 @@ decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
 #pragma unroll
   for (int p = 0; p < PASSES; ++p) s[p] = __ldcs(&state[(size_t)(row0 + p * RPP) * LPR + col4]);
 
-  if (tid < D) {
-    sq[tid] = to_f32<TIn>(q[(size_t)bh * D + tid]);
-    sk[tid] = to_f32<TIn>(k[(size_t)bh * D + tid]);
-  }
-  float4 vv;
-  {
-    const TIn* vp = v + (size_t)bh * E + 4 * col4;
-    vv = make_float4(to_f32<TIn>(vp[0]), to_f32<TIn>(vp[1]), to_f32<TIn>(vp[2]), to_f32<TIn>(vp[3]));
-  }
-  __syncthreads();
-
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-  for (int p = 0; p < PASSES; ++p) {
-    const int i = row0 + p * RPP;
-    const float ki = sk[i], qi = sq[i];
-    float4 x = s[p];
-    x.x = fmaf(lam, x.x, ki * vv.x);
-    x.y = fmaf(lam, x.y, ki * vv.y);
-    x.z = fmaf(lam, x.z, ki * vv.z);
-    x.w = fmaf(lam, x.w, ki * vv.w);
-    __stcs(&state[(size_t)i * LPR + col4], x);
-    acc.x = fmaf(x.x, qi, acc.x);
-    acc.y = fmaf(x.y, qi, acc.y);
-    acc.z = fmaf(x.z, qi, acc.z);
-    acc.w = fmaf(x.w, qi, acc.w);
-  }
-  red[row0][col4] = acc;
-  __syncthreads();
-  if (tid < LPR) {
-    float4 t = red[0][tid];
-#pragma unroll
-    for (int r = 1; r < RPP; ++r) {
-      const float4 u = red[r][tid];
-      t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+  for (int t = 0; t < T; ++t) {
+    if (tid < D) {
+      sq[tid] = to_f32<TIn>(q[((size_t)bh * T + t) * D + tid]);
+      sk[tid] = to_f32<TIn>(k[((size_t)bh * T + t) * D + tid]);
     }
-    TOut* op = o + (size_t)bh * E + 4 * tid;
-    op[0] = from_f32<TOut>(t.x);
-    op[1] = from_f32<TOut>(t.y);
-    op[2] = from_f32<TOut>(t.z);
-    op[3] = from_f32<TOut>(t.w);
+    float4 vv;
+    {
+      const TIn* vp = v + ((size_t)bh * T + t) * E + 4 * col4;
+      vv = make_float4(to_f32<TIn>(vp[0]), to_f32<TIn>(vp[1]), to_f32<TIn>(vp[2]), to_f32<TIn>(vp[3]));
+    }
+    __syncthreads();
+
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) {
+      const int i = row0 + p * RPP;
+      const float ki = sk[i], qi = sq[i];
+      float4 x = s[p];
+      x.x = fmaf(lam, x.x, ki * vv.x);
+      x.y = fmaf(lam, x.y, ki * vv.y);
+      x.z = fmaf(lam, x.z, ki * vv.z);
+      x.w = fmaf(lam, x.w, ki * vv.w);
+      s[p] = x;
+      if (t == T - 1) __stcs(&state[(size_t)i * LPR + col4], x);  // the state leaves once, after the last token
+      acc.x = fmaf(x.x, qi, acc.x);
+      acc.y = fmaf(x.y, qi, acc.y);
+      acc.z = fmaf(x.z, qi, acc.z);
+      acc.w = fmaf(x.w, qi, acc.w);
+    }
+    red[row0][col4] = acc;
+    __syncthreads();
+    if (tid < LPR) {
+      float4 sum = red[0][tid];
+#pragma unroll
+      for (int r = 1; r < RPP; ++r) {
+        const float4 u = red[r][tid];
+        sum.x += u.x; sum.y += u.y; sum.z += u.z; sum.w += u.w;
+      }
+      TOut* op = o + ((size_t)bh * T + t) * E + 4 * tid;
+      op[0] = from_f32<TOut>(sum.x);
+      op[1] = from_f32<TOut>(sum.y);
+      op[2] = from_f32<TOut>(sum.z);
+      op[3] = from_f32<TOut>(sum.w);
+    }
+    // (the next token's q, k are written to sq, sk only after every thread has passed the barrier above; red is
+    // rewritten only after the next barrier)
   }
 }
 
 template <typename TIn, typename TOut, int D, int E>
-cudaError_t launch_t(const void* q, const void* k, const void* v, float* kv, void* o, int BH, int H,
+cudaError_t launch_t(const void* q, const void* k, const void* v, float* kv, void* o, int BH, int H, int T,
                      const DecayTable& tab, cudaStream_t stream) {
   KernelTimer timer(K_DECODE, stream);
   decode_kernel<TIn, TOut, D, E><<<BH, THREADS, 0, stream>>>(
       static_cast<const TIn*>(q), static_cast<const TIn*>(k), static_cast<const TIn*>(v), kv,
-      static_cast<TOut*>(o), H, tab);
+      static_cast<TOut*>(o), H, T, tab);
   count_launch();
   return cudaGetLastError();
 }
 
 template <int D, int E>
-cudaError_t launch_dims(const void* q, const void* k, const void* v, float* kv, void* o, int BH, int H,
+cudaError_t launch_dims(const void* q, const void* k, const void* v, float* kv, void* o, int BH, int H, int T,
                         int in_dt, int out_dt, const DecayTable& tab, cudaStream_t stream) {
   if (in_dt == DT_F32 && out_dt == DT_F32)
-    return launch_t<float, float, D, E>(q, k, v, kv, o, BH, H, tab, stream);
+    return launch_t<float, float, D, E>(q, k, v, kv, o, BH, H, T, tab, stream);
   if (in_dt == DT_BF16 && out_dt == DT_F32)
-    return launch_t<__nv_bfloat16, float, D, E>(q, k, v, kv, o, BH, H, tab, stream);
+    return launch_t<__nv_bfloat16, float, D, E>(q, k, v, kv, o, BH, H, T, tab, stream);
   if (in_dt == DT_BF16 && out_dt == DT_BF16)
-    return launch_t<__nv_bfloat16, __nv_bfloat16, D, E>(q, k, v, kv, o, BH, H, tab, stream);
+    return launch_t<__nv_bfloat16, __nv_bfloat16, D, E>(q, k, v, kv, o, BH, H, T, tab, stream);
   return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv, void* o, int BH,
-                          int H, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
+                          int H, int T, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
                           cudaStream_t stream) {
-  if (d == 64 && e == 64) return launch_dims<64, 64>(q, k, v, kv, o, BH, H, in_dt, out_dt, tab, stream);
+  if (T < 1) return cudaErrorInvalidValue;
+  if (d == 64 && e == 64) return launch_dims<64, 64>(q, k, v, kv, o, BH, H, T, in_dt, out_dt, tab, stream);
   if (d == 128 && e == 128)
-    return launch_dims<128, 128>(q, k, v, kv, o, BH, H, in_dt, out_dt, tab, stream);
+    return launch_dims<128, 128>(q, k, v, kv, o, BH, H, T, in_dt, out_dt, tab, stream);
   return cudaErrorInvalidValue;
 }
 

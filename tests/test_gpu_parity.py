@@ -590,3 +590,31 @@ def test_decode_steps_replay_from_a_cuda_graph():
     graph.replay()
     torch.cuda.synchronize()
     assert torch.equal(kv_graph, kv_eager) and torch.equal(o_graph, o_eager)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("T", [1, 2, 5, 16])
+def test_decode_several_tokens_per_call(T, d):
+    """la_decode_steps: T tokens against the state in one launch equal T single steps bit for bit, and the
+    recurrence of the oracle within tolerance; the state is written once."""
+    B, H = 3, 4
+    lam = torch.tensor([1.0, 0.99, 0.6, 0.05])
+    gen = torch.Generator("cpu")
+    gen.manual_seed(40 + T)
+    q = inputs.draw((B, H, T, d), gen, "silu", torch.bfloat16)
+    k = inputs.draw((B, H, T, d), gen, "silu", torch.bfloat16)
+    v = inputs.draw((B, H, T, d), gen, "normal", torch.bfloat16)
+    kv0 = inputs.make_state(B, H, d, d, seed=41)
+    qg, kg, vg = to_dev(q, k, v)
+    kv_multi = kv0.to(DEV)
+    o_multi = torch.empty((B, H, T, d), dtype=torch.float32, device=DEV)
+    shape = la.make_shape(B, H, T, d, d, torch.bfloat16, torch.float32)
+    la.la_decode_steps(shape, qg, kg, vg, lam, kv_multi, o_multi)
+    kv_single = kv0.to(DEV)
+    outs = [la.decode_step(qg[:, :, t].contiguous(), kg[:, :, t].contiguous(), vg[:, :, t].contiguous(), lam, kv_single)
+            for t in range(T)]
+    torch.cuda.synchronize()
+    assert torch.equal(o_multi, torch.stack(outs, dim=2)) and torch.equal(kv_multi, kv_single)
+    ref_o, ref_kv = orc.fwd_rec(q, k, v, lam.double().numpy(), kv_in=kv0.double().numpy(), want_state=True)
+    assert_close(o_multi, ref_o, 1e-5, "o")
+    assert_close(kv_multi, ref_kv, 1e-5, "state")
