@@ -16,8 +16,8 @@
  *
  * Conventions that hold for every entry point
  *   - Tensors are dense row-major with the feature dimension fastest:
- *     q,k,dq,dk [B,H,N,d]; v,o,dO,dv [B,H,N,e]; states [B,H,d,e] fp32 with
- *     kv[b,h,i,j] = sum_s lambda^(t-s) k_s[i] v_s[j].
+ *     q,k,dq,dk [B,H,N,d]; v,o,dO,dv [B,H,N,e] (or [B,N,H,.] with la_shape.layout =
+ *     LA_LAYOUT_BNHD); states [B,H,d,e] fp32 with kv[b,h,i,j] = sum_s lambda^(t-s) k_s[i] v_s[j].
  *   - Every tensor pointer is DEVICE memory, 16-byte aligned, owned by the caller.
  *     The library allocates no device memory, never frees and never synchronises
  *     the stream (la_device_status and la_profile_collect are the two calls that
@@ -79,6 +79,12 @@ typedef enum { LA_PATH_AUTO = 0, LA_PATH_SIMT = 1, LA_PATH_TENSOR = 2 } la_path;
 #define LA_SPLIT_DECAYED 4 /* the decay-scaled value rows entering the state update  */
 #define LA_PRECISION_DEFAULT (-1)
 
+/* Layout of the token tensors (q, k, v, dO, o, dq, dk, dv, u, y): feature dimension always fastest.
+ * LA_LAYOUT_BHND: [B,H,N,d] as in the operation's definition.  LA_LAYOUT_BNHD: [B,N,H,d], the layout a fused
+ * Q/K/V/U projection of the token mixer leaves its output in (Eq. 3: the heads of one token are adjacent); rstd
+ * follows as [B,N,H].  States are [B,H,d,e] in both.  la_fwd_bwd_host takes LA_LAYOUT_BHND only. */
+typedef enum { LA_LAYOUT_BHND = 0, LA_LAYOUT_BNHD = 1 } la_layout;
+
 typedef struct {
   int B, H, N, d, e;  /* N >= 1 (ignored by la_decode_step) */
   la_dtype in_dtype;  /* q, k, v, dO */
@@ -88,6 +94,7 @@ typedef struct {
                          that run as independent thread blocks joined by a state scan. */
   int path;           /* la_path */
   int precision;      /* LA_PRECISION_DEFAULT or an OR of LA_SPLIT_* */
+  int layout;         /* la_layout */
 } la_shape;
 
 #define LA_OP_FWD 0

@@ -21,6 +21,7 @@ LA_PATH_AUTO, LA_PATH_SIMT, LA_PATH_TENSOR = 0, 1, 2
 LA_SPLIT_SCORES, LA_SPLIT_STATE, LA_SPLIT_DECAYED = 1, 2, 4
 LA_PRECISION_DEFAULT = -1
 LA_OP_FWD, LA_OP_BWD, LA_OP_DECODE = 0, 1, 2
+LA_LAYOUT_BHND, LA_LAYOUT_BNHD = 0, 1
 
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
@@ -33,7 +34,8 @@ KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate")
 class LaShape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int), ("H", ctypes.c_int), ("N", ctypes.c_int), ("d", ctypes.c_int),
                 ("e", ctypes.c_int), ("in_dtype", ctypes.c_int), ("out_dtype", ctypes.c_int),
-                ("seg_len", ctypes.c_int), ("path", ctypes.c_int), ("precision", ctypes.c_int)]
+                ("seg_len", ctypes.c_int), ("path", ctypes.c_int), ("precision", ctypes.c_int),
+                ("layout", ctypes.c_int)]
 
 
 class LaError(RuntimeError):
@@ -145,8 +147,8 @@ _DT = {torch.bfloat16: LA_BF16, torch.float32: LA_F32}
 
 
 def make_shape(B, H, N, d, e, in_dtype, out_dtype, seg_len=0, path=LA_PATH_AUTO,
-               precision=LA_PRECISION_DEFAULT) -> LaShape:
-    return LaShape(B, H, N, d, e, _DT[in_dtype], _DT[out_dtype], seg_len, path, precision)
+               precision=LA_PRECISION_DEFAULT, layout=LA_LAYOUT_BHND) -> LaShape:
+    return LaShape(B, H, N, d, e, _DT[in_dtype], _DT[out_dtype], seg_len, path, precision, layout)
 
 
 def workspace_bytes(op: int, shape: LaShape) -> int:

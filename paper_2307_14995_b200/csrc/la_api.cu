@@ -58,6 +58,7 @@ la_status check_shape(const la_shape* s, bool need_n) {
   if (s->path < LA_PATH_AUTO || s->path > LA_PATH_TENSOR) return LA_ERR_INVALID_ARG;
   if (s->precision != LA_PRECISION_DEFAULT && (s->precision < 0 || s->precision > 7))
     return LA_ERR_INVALID_ARG;
+  if (s->layout != LA_LAYOUT_BHND && s->layout != LA_LAYOUT_BNHD) return LA_ERR_INVALID_ARG;
   if (s->H > LA_MAX_H) return LA_ERR_UNSUPPORTED;
   if (!(s->d == s->e && (s->d == 64 || s->d == 128))) return LA_ERR_UNSUPPORTED;
   if (s->in_dtype == LA_F32 && s->out_dtype != LA_F32) return LA_ERR_UNSUPPORTED;
@@ -152,6 +153,20 @@ struct OpCall {
   float* buf;            // [BH,nseg,D*E] scratch for entry states (may be NULL if not needed)
 };
 
+// Element strides of the token tensors for the shape's layout (d == e in every supported shape).
+void set_strides(const la_shape* s, int tokens, OpArgs* a) {
+  const long long D = s->d;
+  if (s->layout == LA_LAYOUT_BNHD) {
+    a->sT = (long long)s->H * D;
+    a->sH = D;
+    a->sB = (long long)tokens * s->H * D;
+  } else {
+    a->sT = D;
+    a->sH = (long long)tokens * D;
+    a->sB = (long long)s->H * tokens * D;
+  }
+}
+
 cudaError_t run_prepass(const la_shape* s, const Plan& p, const DecayTable& tab, const void* b,
                         const void* c, int reverse, float* local_out, cudaStream_t st) {
   OpArgs args{};
@@ -164,6 +179,7 @@ cudaError_t run_prepass(const la_shape* s, const Plan& p, const DecayTable& tab,
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
+  set_strides(s, s->N, &args);
   if (p.tensor) return launch_tc_prepass(args, tab, s->d, p.precision, st);
   return launch_simt_prepass(args, tab, s->d, s->e, (int)s->in_dtype, st);
 }
@@ -201,6 +217,7 @@ OpArgs walk_args(const la_shape* s, const Plan& p, const void* a, const void* b,
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
+  set_strides(s, s->N, &args);
   return args;
 }
 
@@ -433,8 +450,10 @@ la_status decode_impl(const la_shape* shape, int T, const void* q, const void* k
   DecayTable tab;
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
   if ((st = check_device()) != LA_OK) return st;
+  OpArgs strides{};
+  set_strides(shape, T, &strides);
   LA_TRY_CUDA(launch_decode(q, k, v, kv, o, shape->B * shape->H, shape->H, T, shape->d, shape->e,
-                            (int)shape->in_dtype, (int)shape->out_dtype, tab,
+                            (int)shape->in_dtype, (int)shape->out_dtype, strides.sT, strides.sH, strides.sB, tab,
                             static_cast<cudaStream_t>(stream)));
   return LA_OK;
 }
@@ -496,6 +515,7 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
                           void* device_arena, size_t arena_bytes, void* stream) {
   const size_t need = la_host_arena_bytes(shape);
   if (need == (size_t)-1) return check_shape(shape, true) != LA_OK ? check_shape(shape, true) : LA_ERR_UNSUPPORTED;
+  if (shape->layout != LA_LAYOUT_BHND) return LA_ERR_UNSUPPORTED;  // the head groups must be contiguous slices
   if (!q_host || !k_host || !v_host || !d_o_host || !o_host || !dq_host || !dk_host || !dv_host)
     return LA_ERR_INVALID_ARG;
   if (!device_arena || arena_bytes < need) return LA_ERR_WORKSPACE;

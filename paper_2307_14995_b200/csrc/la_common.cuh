@@ -48,6 +48,10 @@ struct OpArgs {
   int BH, H, N;
   int seg_len, nseg;  // seg_len is a multiple of 128
   int reverse;        // 0 forward, 1 reverse
+  // Where token t of (batch b, head h) sits in a, b, c, out, u, y: element offset b*sB + h*sH + t*sT of a row of
+  // Da / Ec contiguous features.  [B,H,N,D]: sT = D, sH = N*D, sB = H*N*D; [B,N,H,D]: sT = H*D, sH = D, sB = N*H*D
+  // (D = Da = Ec in every supported shape).
+  long long sT, sH, sB;
   // Optional epilogue of the forward walk (Eq. 3 with Eq. 8): y = SRMSNorm(out) (.) u per row.  With u set, y is
   // written, `out` becomes optional (NULL = the attention output itself is not wanted) and rstd [BH, N] optional.
   const void* u;      // [BH, N, Ec] gate, input dtype
@@ -74,10 +78,10 @@ cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int D
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream);
 // dst[m] = transpose(src[m]) for `count` row-major Da x Ec fp32 matrices.
 cudaError_t launch_transpose_states(const float* src, float* dst, long count, int Da, int Ec, cudaStream_t stream);
-// T >= 1 consecutive tokens per (batch, head): q, k [BH, T, d], v, o [BH, T, e].
+// T >= 1 consecutive tokens per (batch, head); token t of (b,h) is the row at element offset b*sB + h*sH + t*sT.
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv, void* o, int BH,
-                          int H, int T, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
-                          cudaStream_t stream);
+                          int H, int T, int d, int e, int in_dt, int out_dt, long long sT, long long sH, long long sB,
+                          const DecayTable& tab, cudaStream_t stream);
 
 // SimpleRMSNorm followed by the gate as stand-alone row kernels (la_gate.cu): y = SRMSNorm(o) (.) u (o and y may be
 // the same buffer), and the gradients of <y, dy> with respect to o (written in the input dtype) and u.

@@ -20,7 +20,8 @@ constexpr int THREADS = 256;
 template <typename TIn, typename TOut, int D, int E>
 __global__ void __launch_bounds__(THREADS)
 decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* __restrict__ v,
-              float* __restrict__ kv, TOut* __restrict__ o, int H, int T, const DecayTable tab) {
+              float* __restrict__ kv, TOut* __restrict__ o, int H, int T, long long sT, long long sH, long long sB,
+              const DecayTable tab) {
   constexpr int LPR = E / 4;              // lanes per state row (float4 each)
   constexpr int RPP = THREADS / LPR;      // rows per pass
   constexpr int PASSES = D / RPP;
@@ -37,6 +38,7 @@ decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
   const int row0 = tid / LPR;
 
   float4* state = reinterpret_cast<float4*>(kv + (size_t)bh * D * E);
+  const size_t head_off = (size_t)(bh / H) * sB + (size_t)(bh % H) * sH;  // token t of this (b,h): + t * sT
 
   // issue every state load first: PASSES independent 16-byte loads per thread
   float4 s[PASSES];
@@ -45,12 +47,12 @@ decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
 
   for (int t = 0; t < T; ++t) {
     if (tid < D) {
-      sq[tid] = to_f32<TIn>(q[((size_t)bh * T + t) * D + tid]);
-      sk[tid] = to_f32<TIn>(k[((size_t)bh * T + t) * D + tid]);
+      sq[tid] = to_f32<TIn>(q[head_off + (size_t)t * sT + tid]);
+      sk[tid] = to_f32<TIn>(k[head_off + (size_t)t * sT + tid]);
     }
     float4 vv;
     {
-      const TIn* vp = v + ((size_t)bh * T + t) * E + 4 * col4;
+      const TIn* vp = v + head_off + (size_t)t * sT + 4 * col4;
       vv = make_float4(to_f32<TIn>(vp[0]), to_f32<TIn>(vp[1]), to_f32<TIn>(vp[2]), to_f32<TIn>(vp[3]));
     }
     __syncthreads();
@@ -81,7 +83,7 @@ decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
         const float4 u = red[r][tid];
         sum.x += u.x; sum.y += u.y; sum.z += u.z; sum.w += u.w;
       }
-      TOut* op = o + ((size_t)bh * T + t) * E + 4 * tid;
+      TOut* op = o + head_off + (size_t)t * sT + 4 * tid;
       op[0] = from_f32<TOut>(sum.x);
       op[1] = from_f32<TOut>(sum.y);
       op[2] = from_f32<TOut>(sum.z);
@@ -94,36 +96,37 @@ decode_kernel(const TIn* __restrict__ q, const TIn* __restrict__ k, const TIn* _
 
 template <typename TIn, typename TOut, int D, int E>
 cudaError_t launch_t(const void* q, const void* k, const void* v, float* kv, void* o, int BH, int H, int T,
-                     const DecayTable& tab, cudaStream_t stream) {
+                     long long sT, long long sH, long long sB, const DecayTable& tab, cudaStream_t stream) {
   KernelTimer timer(K_DECODE, stream);
   decode_kernel<TIn, TOut, D, E><<<BH, THREADS, 0, stream>>>(
       static_cast<const TIn*>(q), static_cast<const TIn*>(k), static_cast<const TIn*>(v), kv,
-      static_cast<TOut*>(o), H, T, tab);
+      static_cast<TOut*>(o), H, T, sT, sH, sB, tab);
   count_launch();
   return cudaGetLastError();
 }
 
 template <int D, int E>
 cudaError_t launch_dims(const void* q, const void* k, const void* v, float* kv, void* o, int BH, int H, int T,
-                        int in_dt, int out_dt, const DecayTable& tab, cudaStream_t stream) {
+                        int in_dt, int out_dt, long long sT, long long sH, long long sB, const DecayTable& tab,
+                        cudaStream_t stream) {
   if (in_dt == DT_F32 && out_dt == DT_F32)
-    return launch_t<float, float, D, E>(q, k, v, kv, o, BH, H, T, tab, stream);
+    return launch_t<float, float, D, E>(q, k, v, kv, o, BH, H, T, sT, sH, sB, tab, stream);
   if (in_dt == DT_BF16 && out_dt == DT_F32)
-    return launch_t<__nv_bfloat16, float, D, E>(q, k, v, kv, o, BH, H, T, tab, stream);
+    return launch_t<__nv_bfloat16, float, D, E>(q, k, v, kv, o, BH, H, T, sT, sH, sB, tab, stream);
   if (in_dt == DT_BF16 && out_dt == DT_BF16)
-    return launch_t<__nv_bfloat16, __nv_bfloat16, D, E>(q, k, v, kv, o, BH, H, T, tab, stream);
+    return launch_t<__nv_bfloat16, __nv_bfloat16, D, E>(q, k, v, kv, o, BH, H, T, sT, sH, sB, tab, stream);
   return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
 cudaError_t launch_decode(const void* q, const void* k, const void* v, float* kv, void* o, int BH,
-                          int H, int T, int d, int e, int in_dt, int out_dt, const DecayTable& tab,
-                          cudaStream_t stream) {
+                          int H, int T, int d, int e, int in_dt, int out_dt, long long sT, long long sH, long long sB,
+                          const DecayTable& tab, cudaStream_t stream) {
   if (T < 1) return cudaErrorInvalidValue;
-  if (d == 64 && e == 64) return launch_dims<64, 64>(q, k, v, kv, o, BH, H, T, in_dt, out_dt, tab, stream);
+  if (d == 64 && e == 64) return launch_dims<64, 64>(q, k, v, kv, o, BH, H, T, in_dt, out_dt, sT, sH, sB, tab, stream);
   if (d == 128 && e == 128)
-    return launch_dims<128, 128>(q, k, v, kv, o, BH, H, T, in_dt, out_dt, tab, stream);
+    return launch_dims<128, 128>(q, k, v, kv, o, BH, H, T, in_dt, out_dt, sT, sH, sB, tab, stream);
   return cudaErrorInvalidValue;
 }
 

@@ -33,19 +33,20 @@ struct Smem {
 };
 
 template <typename TIn, int W>
-__device__ __forceinline__ void load_tile_natural(float (*dst)[W], const TIn* src, int rows_valid) {
-  // dst[i][k] = src[i*W + k] for i < rows_valid, else 0
+__device__ __forceinline__ void load_tile_natural(float (*dst)[W], const TIn* src, long long row_stride, int rows_valid) {
+  // dst[i][k] = src[i*row_stride + k] for i < rows_valid, else 0
   for (int idx = threadIdx.x; idx < C * W; idx += THREADS) {
     const int i = idx / W, k = idx % W;
-    dst[i][k] = (i < rows_valid) ? to_f32<TIn>(src[(size_t)i * W + k]) : 0.f;
+    dst[i][k] = (i < rows_valid) ? to_f32<TIn>(src[(size_t)i * row_stride + k]) : 0.f;
   }
 }
 
 template <typename TIn, int W>
-__device__ __forceinline__ void load_tile_transposed(float (*dstT)[AP], const TIn* src, int rows_valid) {
+__device__ __forceinline__ void load_tile_transposed(float (*dstT)[AP], const TIn* src, long long row_stride,
+                                                     int rows_valid) {
   for (int idx = threadIdx.x; idx < C * W; idx += THREADS) {
     const int i = idx / W, k = idx % W;
-    dstT[k][i] = (i < rows_valid) ? to_f32<TIn>(src[(size_t)i * W + k]) : 0.f;
+    dstT[k][i] = (i < rows_valid) ? to_f32<TIn>(src[(size_t)i * row_stride + k]) : 0.f;
   }
 }
 
@@ -63,10 +64,12 @@ simt_walk_kernel(const OpArgs args, const DecayTable tab) {
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
   const int nblk = (seg_t1 - seg_t0 + C - 1) / C;
 
-  const TIn* a = static_cast<const TIn*>(args.a) + (size_t)bh * args.N * DA;
-  const TIn* b = static_cast<const TIn*>(args.b) + (size_t)bh * args.N * DA;
-  const TIn* c = static_cast<const TIn*>(args.c) + (size_t)bh * args.N * EC;
-  TOut* out = static_cast<TOut*>(args.out) + (size_t)bh * args.N * EC;
+  const size_t head_off = (size_t)(bh / args.H) * args.sB + (size_t)(bh % args.H) * args.sH;
+  const long long sT = args.sT;  // elements between consecutive tokens
+  const TIn* a = static_cast<const TIn*>(args.a) + head_off;
+  const TIn* b = static_cast<const TIn*>(args.b) + head_off;
+  const TIn* c = static_cast<const TIn*>(args.c) + head_off;
+  TOut* out = static_cast<TOut*>(args.out) + head_off;
 
   // state entering this segment
   {
@@ -92,10 +95,10 @@ simt_walk_kernel(const OpArgs args, const DecayTable tab) {
       }
       if (i == 0) sm.gamma = decay_pow_d(s2, (double)Cr);
     }
-    load_tile_transposed<TIn, DA>(sm.aT, a + (size_t)t0 * DA, Cr);
-    load_tile_transposed<TIn, DA>(sm.bT, b + (size_t)t0 * DA, Cr);
-    load_tile_natural<TIn, DA>(sm.b, b + (size_t)t0 * DA, Cr);
-    load_tile_natural<TIn, EC>(sm.c, c + (size_t)t0 * EC, Cr);
+    load_tile_transposed<TIn, DA>(sm.aT, a + (size_t)t0 * sT, sT, Cr);
+    load_tile_transposed<TIn, DA>(sm.bT, b + (size_t)t0 * sT, sT, Cr);
+    load_tile_natural<TIn, DA>(sm.b, b + (size_t)t0 * sT, sT, Cr);
+    load_tile_natural<TIn, EC>(sm.c, c + (size_t)t0 * sT, sT, Cr);
     __syncthreads();
 
     // (1) masked scores: pT[j][i] = (a_i . b_j) * D_ij
@@ -164,7 +167,7 @@ simt_walk_kernel(const OpArgs args, const DecayTable tab) {
           const float f = sm.f_out[i];
 #pragma unroll
           for (int m = 0; m < EM; ++m)
-            out[(size_t)(t0 + i) * EC + tx + 32 * m] = from_f32<TOut>(fmaf(f, inter[r][m], intra[r][m]));
+            out[(size_t)(t0 + i) * sT + tx + 32 * m] = from_f32<TOut>(fmaf(f, inter[r][m], intra[r][m]));
         }
       }
     }
@@ -234,8 +237,10 @@ simt_prepass_kernel(const OpArgs args, const DecayTable tab) {
   const int seg_t0 = seg * args.seg_len;
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
   const int nblk = (seg_t1 - seg_t0 + C - 1) / C;
-  const TIn* b = static_cast<const TIn*>(args.b) + (size_t)bh * args.N * DA;
-  const TIn* c = static_cast<const TIn*>(args.c) + (size_t)bh * args.N * EC;
+  const size_t head_off = (size_t)(bh / args.H) * args.sB + (size_t)(bh % args.H) * args.sH;
+  const long long sT = args.sT;
+  const TIn* b = static_cast<const TIn*>(args.b) + head_off;
+  const TIn* c = static_cast<const TIn*>(args.c) + head_off;
 
   constexpr int RK = DA / 16, RE = EC / 16;
   const int ty = tid / 16, tx = tid % 16;
@@ -254,8 +259,8 @@ simt_prepass_kernel(const OpArgs args, const DecayTable tab) {
       if (tid < Cr) f = REV ? decay_pow_d(s2, (double)(t - seg_t0 + 1)) : decay_pow_d(s2, (double)(seg_t1 - 1 - t));
       sm.f_state[tid] = f;
     }
-    load_tile_natural<TIn, DA>(sm.b, b + (size_t)t0 * DA, Cr);
-    load_tile_natural<TIn, EC>(sm.c, c + (size_t)t0 * EC, Cr);
+    load_tile_natural<TIn, DA>(sm.b, b + (size_t)t0 * sT, sT, Cr);
+    load_tile_natural<TIn, EC>(sm.c, c + (size_t)t0 * sT, sT, Cr);
     __syncthreads();
 #pragma unroll 2
     for (int j = 0; j < C; ++j) {

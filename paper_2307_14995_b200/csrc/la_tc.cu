@@ -120,6 +120,7 @@ struct TcArgs {
   int njobs;
   int BH, H, N, seg_len, nseg;
   int precision;
+  long long sT, sH, sB;  // element offset of token t of (b,h): b*sB + h*sH + t*sT (rows of D contiguous features)
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
@@ -245,6 +246,8 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
   const int ehalf = (D == 128) ? (int)(bidx & 1) : 0;
   const int segid = (D == 128) ? (int)(bidx >> 1) : (int)bidx;
   const int bh = segid / args.nseg, seg = segid % args.nseg;
+  const int hh_ = bh % args.H, bb_ = bh / args.H;  // head and batch coordinates of the 4-D tensor maps
+  const size_t head_off = (size_t)bb_ * args.sB + (size_t)hh_ * args.sH;
   const int seg_t0 = seg * args.seg_len;
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
   const float s2 = (float)tab.s2[bh % args.H];
@@ -326,29 +329,29 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
         // (measured: 0.276 -> 0.245 ms per launch; the same in the walk kernel made it slower).
         if (STATE_ONLY && it + 2 < nblk) {
           const int tp = seg_t0 + (REV ? (nblk - 3 - it) : (it + 2 + it0)) * 128;
-          tma_prefetch_3d(tm_b, 0, tp, bh);
-          if (D == 128) tma_prefetch_3d(tm_b, 64, tp, bh);
-          tma_prefetch_3d(tm_c, ehalf * 64, tp, bh);
+          tma_prefetch_4d(tm_b, 0, tp, hh_, bb_);
+          if (D == 128) tma_prefetch_4d(tm_b, 64, tp, hh_, bb_);
+          tma_prefetch_4d(tm_c, ehalf * 64, tp, hh_, bb_);
         }
         if (STATE_ONLY) {
           if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
           mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 256);
-          tma_load_3d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
+          tma_load_4d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, hh_, bb_);
+          if (D == 128) tma_load_4d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, hh_, bb_);
         } else {
           // walk kernel: the a and b tiles of a stage travel together (one barrier for both, FULL_B); A_FREE
           // is committed after M2, the last product of the block that reads either of them
           if (it >= 2) TC_WAIT(A_FREE0 + s, prev, 3);
           mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 512);
-          tma_load_3d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, bh);
-          tma_load_3d(&stg.a[0][0], tm_a, &sm.bars[FULL_B0 + s], 0, t0, bh);
-          if (D == 128) tma_load_3d(&stg.a[1][0], tm_a, &sm.bars[FULL_B0 + s], 64, t0, bh);
+          tma_load_4d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, hh_, bb_);
+          if (D == 128) tma_load_4d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, hh_, bb_);
+          tma_load_4d(&stg.a[0][0], tm_a, &sm.bars[FULL_B0 + s], 0, t0, hh_, bb_);
+          if (D == 128) tma_load_4d(&stg.a[1][0], tm_a, &sm.bars[FULL_B0 + s], 64, t0, hh_, bb_);
         }
         armed_b[s] = (it >> 1) + 1;
         if (it >= 2) TC_WAIT(C_FREE0 + s, prev, 2);
         mbar_arrive_expect_tx(&sm.bars[FULL_C0 + s], 16384);
-        tma_load_3d(&stg.c[0], tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, bh);
+        tma_load_4d(&stg.c[0], tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, hh_, bb_);
         armed_c[s] = (it >> 1) + 1;
       }
     }
@@ -606,11 +609,11 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
     auto c_from_global = [&](int it, uint4 (&raw)[4]) {
       const int blk = REV ? (nblk - 1 - it) : it;
       const int t0 = seg_t0 + blk * 128;
-      const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
-                                                        ((size_t)bh * args.N + t0 + frow) * D + ehalf * 64) + fch;
+      const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(job.c) + head_off + (size_t)(t0 + frow) * args.sT +
+                                 ehalf * 64 + fch * 8;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(src + (size_t)i * 32 * (D / 8));  // 32 rows of D / 8 chunks on
+        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(32 * i) * args.sT));
         else raw[i] = make_uint4(0u, 0u, 0u, 0u);
       }
     };
@@ -756,7 +759,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
           ++og_uses;
           if (warp == 20 && lane == 0) {
             // rows beyond N are clipped by the tensor map (a ragged block is always the last of the sequence)
-            tma_store_3d(tm_out, stg, ehalf * 64 + pass * (int)(128 / sizeof(TOut)), t0, bh);
+            tma_store_4d(tm_out, stg, ehalf * 64 + pass * (int)(128 / sizeof(TOut)), t0, hh_, bb_);
             tma_store_commit();
           }
         }
@@ -824,17 +827,19 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over a [BH, N, D] tensor (feature dimension innermost, D = 64 or 128) of bf16 or fp32 with a box of
-// 128 bytes x 128 rows x 1 and 128-byte swizzle; rows beyond N read as zero and are not written.
-bool make_map(CUtensorMap* m, const void* ptr, int N, int BH, int D, bool f32 = false) {
+// Tensor map over a token tensor seen as {feature D, token N, head H, batch B} with element strides {1, sT, sH, sB}
+// (D = 64 or 128, bf16 or fp32), a box of 128 bytes x 128 tokens x 1 x 1 and 128-byte swizzle; tokens beyond N read
+// as zero and are not written.
+bool make_map(CUtensorMap* m, const void* ptr, const OpArgs& a, int D, bool f32 = false) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   const cuuint64_t esz = f32 ? 4 : 2;
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)N, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {D * esz, (cuuint64_t)N * D * esz};
-  cuuint32_t box[3] = {(cuuint32_t)(128 / esz), 128, 1};
-  cuuint32_t es[3] = {1, 1, 1};
-  return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr),
+  const int B = a.BH / a.H;
+  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)a.N, (cuuint64_t)a.H, (cuuint64_t)B};
+  cuuint64_t strides[3] = {(cuuint64_t)a.sT * esz, (cuuint64_t)a.sH * esz, (cuuint64_t)a.sB * esz};
+  cuuint32_t box[4] = {(cuuint32_t)(128 / esz), 128, 1, 1};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr),
              dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -852,9 +857,8 @@ cudaError_t launch_t(const TcMaps& m0, const TcMaps& m1, const TcArgs& ta, const
 }
 
 bool make_maps(TcMaps* m, const OpArgs& args, int D, bool f32) {
-  return make_map(&m->a, args.a, args.N, args.BH, D) && make_map(&m->b, args.b, args.N, args.BH, D) &&
-         make_map(&m->c, args.c, args.N, args.BH, D) &&
-         make_map(&m->out, args.out ? args.out : args.y, args.N, args.BH, D, f32);  // (gated walk without `out`: y)
+  return make_map(&m->a, args.a, args, D) && make_map(&m->b, args.b, args, D) && make_map(&m->c, args.c, args, D) &&
+         make_map(&m->out, args.out ? args.out : args.y, args, D, f32);  // (gated walk without `out`: y)
 }
 
 // One walk (second == nullptr) or two walks of the same direction over the same tokens in one launch.
@@ -876,6 +880,7 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   ta.njobs = second ? 2 : 1;
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
+  ta.sT = args.sT; ta.sH = args.sH; ta.sB = args.sB;
   if (args.u) {
     // forward walk with the gate epilogue: only the full-width kernel has it (the caller asks tc_can_fuse_gate first)
     if (D != 128 || second || args.reverse || !tc_can_fuse_gate(args, D)) return cudaErrorInvalidValue;
@@ -913,7 +918,7 @@ template <int D>
 cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int precision, cudaStream_t stream) {
   TcMaps m;
   // the a and out maps are unused by the state-only kernel; valid descriptors are passed anyway
-  if (!make_map(&m.b, args.b, args.N, args.BH, D) || !make_map(&m.c, args.c, args.N, args.BH, D))
+  if (!make_map(&m.b, args.b, args, D) || !make_map(&m.c, args.c, args, D))
     return cudaErrorInvalidValue;
   m.a = m.b;
   m.out = m.c;
@@ -924,6 +929,7 @@ cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int prec
   ta.njobs = 1;
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
+  ta.sT = args.sT; ta.sH = args.sH; ta.sB = args.sB;
   return args.reverse ? launch_t<true, true, float, D, 1>(m, m, ta, tab, stream)
                       : launch_t<false, true, float, D, 1>(m, m, ta, tab, stream);
 }

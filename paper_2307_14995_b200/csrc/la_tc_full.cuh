@@ -85,6 +85,8 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
   if (NJOBS == 2 && jobid) job = args.job[1];
   const TcMaps& maps = (NJOBS == 2 && jobid) ? maps1 : maps0;
   const int bh = bidx / args.nseg, seg = bidx % args.nseg;
+  const int hh_ = bh % args.H, bb_ = bh / args.H;  // head and batch coordinates of the 4-D tensor maps
+  const size_t head_off = (size_t)bb_ * args.sB + (size_t)hh_ * args.sH;
   const int seg_t0 = seg * args.seg_len;
   const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
   const int nblk = (seg_t1 - seg_t0 + 127) >> 7;
@@ -131,17 +133,17 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
           // reloaded as soon as it falls free; both count towards the one barrier M1 of this block waits for
           if (it >= 1) TC_WAIT(F_DZ_READY, (it - 1) & 1, 3);
           mbar_arrive_expect_tx(&sm.bars[F_FULL_AB], 32768);
-          tma_load_3d(&sm.b[0][0], &maps.b, &sm.bars[F_FULL_AB], 0, t0, bh);
-          tma_load_3d(&sm.b[1][0], &maps.b, &sm.bars[F_FULL_AB], 64, t0, bh);
+          tma_load_4d(&sm.b[0][0], &maps.b, &sm.bars[F_FULL_AB], 0, t0, hh_, bb_);
+          tma_load_4d(&sm.b[1][0], &maps.b, &sm.bars[F_FULL_AB], 64, t0, hh_, bb_);
           if (it >= 1) TC_WAIT(F_AB_FREE, (it - 1) & 1, 5);
           mbar_arrive_expect_tx(&sm.bars[F_FULL_AB], 32768);
-          tma_load_3d(&sm.a[0][0], &maps.a, &sm.bars[F_FULL_AB], 0, t0, bh);
-          tma_load_3d(&sm.a[1][0], &maps.a, &sm.bars[F_FULL_AB], 64, t0, bh);
+          tma_load_4d(&sm.a[0][0], &maps.a, &sm.bars[F_FULL_AB], 0, t0, hh_, bb_);
+          tma_load_4d(&sm.a[1][0], &maps.a, &sm.bars[F_FULL_AB], 64, t0, hh_, bb_);
           armed_ab = it + 1;
           if (it >= 1) TC_WAIT(F_O_READY, (it - 1) & 1, 2);
           mbar_arrive_expect_tx(&sm.bars[F_M4_OK], 32768);
-          tma_load_3d(&sm.c[0][0], &maps.c, &sm.bars[F_M4_OK], 0, t0, bh);
-          tma_load_3d(&sm.c[1][0], &maps.c, &sm.bars[F_M4_OK], 64, t0, bh);
+          tma_load_4d(&sm.c[0][0], &maps.c, &sm.bars[F_M4_OK], 0, t0, hh_, bb_);
+          tma_load_4d(&sm.c[1][0], &maps.c, &sm.bars[F_M4_OK], 64, t0, hh_, bb_);
           armed_c = it + 1;
         }
       }
@@ -291,11 +293,10 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
     // this thread's four pieces of c straight from global memory; rows beyond N read as zero
     auto c_from_global = [&](int it, uint4 (&raw)[4]) {
       const int t0 = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;
-      const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.c) +
-                                                        ((size_t)bh * args.N + t0 + frow) * 128) + fch;
+      const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(job.c) + head_off + (size_t)(t0 + frow) * args.sT + fch * 8;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(src + (size_t)i * 32 * 16);  // 32 rows of 16 chunks on
+        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(32 * i) * args.sT));
         else raw[i] = make_uint4(0u, 0u, 0u, 0u);
       }
     };
@@ -393,9 +394,9 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
       const int Cr = min(128, seg_t1 - t0);
       float f = 0.f;
       if (r < Cr) f = REV ? ex2_approx(-s2 * (float)(Cr - 1 - r)) : ex2_approx(-s2 * (float)(r + 1));
-      // byte address of column 32 g / 4 .. of this thread's own row; the other rows of the quad are 512 or 256 bytes apart
-      unsigned char* const quad_base =
-          static_cast<unsigned char*>(job.out) + ((size_t)bh * args.N + t0 + (r & ~3)) * 128 * sizeof(TOut) + g * 32;
+      // element offset of the first row of this thread's quad; the other rows are sT elements apart
+      const size_t quad_row0 = head_off + (size_t)(t0 + (r & ~3)) * args.sT;
+      unsigned char* const quad_base = static_cast<unsigned char*>(job.out) + quad_row0 * sizeof(TOut) + g * 32;
       // O_READY: every product up to M4 of this block is done
       TC_WAIT_WARP(F_O_READY, it & 1, 25);
       tc_fence_after_sync();
@@ -417,7 +418,8 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
           }
         }
         const float s = ss > 0.f ? rsqrtf(ss * (1.f / 128.f)) : 0.f;
-        if (job.rstd && ohalf == 0 && r < Cr) job.rstd[(size_t)bh * args.N + t0 + r] = s;
+        // rstd has the layout of the token tensors without the feature dimension
+        if (job.rstd && ohalf == 0 && r < Cr) job.rstd[(head_off + (size_t)(t0 + r) * args.sT) >> 7] = s;
 #pragma unroll
         for (int k = 0; k < 4; ++k) srow[k] = __shfl_xor_sync(0xffffffffu, s, k);
       }
@@ -476,10 +478,10 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
           const int row_in_quad = g ^ k;  // slot k holds the row of lane ^ k
           if ((r & ~3) + row_in_quad >= Cr) continue;
           if (!GATED) {
-            st_global_v8(quad_base + (size_t)row_in_quad * (128 * sizeof(TOut)) + pc * 128, &w[8 * k]);
+            st_global_v8(quad_base + (size_t)row_in_quad * args.sT * sizeof(TOut) + pc * 128, &w[8 * k]);
           } else {
             // slot k: columns pc * 32 + 8 g .. + 8 of that row, still fp32
-            const size_t elem = ((size_t)bh * args.N + t0 + (r & ~3) + row_in_quad) * 128 + pc * 32 + g * 8;
+            const size_t elem = quad_row0 + (size_t)row_in_quad * args.sT + pc * 32 + g * 8;
             const uint4 uraw = __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(job.u) + elem));
             const uint32_t uw[4] = {uraw.x, uraw.y, uraw.z, uraw.w};
             uint32_t yv[8];

@@ -193,3 +193,26 @@ def test_gated_forward_then_backward_chain():
     ref_dq, ref_dk, ref_dv = orc.bwd_rec(q, k, v, d_o.cpu(), lam64)
     for n, g, r in (("dq", dq, ref_dq), ("dk", dk, ref_dk), ("dv", dv, ref_dv)):
         assert_close(g, r, TOL_BF16, n)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_gated_forward_token_major_layout(d):
+    """[B,N,H,d] tensors (q, k, v, u as a fused projection leaves them; y, o and rstd [B,N,H] in the same order)."""
+    B, H, N = 2, 3, 650
+    q, k, v, _ = inputs.make_qkvdo(B, H, N, d, d, seed=81, with_do=False)
+    u = draw_gate((B, H, N, d), seed=82)
+    lam = torch.tensor([1.0, 0.97, 0.3])
+    ref_o = orc.fwd_rec(q, k, v, lam.double().numpy())
+    ref_y, ref_rstd = orc.norm_gate_fwd(ref_o, u, want_rstd=True)
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(DEV)
+    shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, 256, layout=la.LA_LAYOUT_BNHD)
+    y, o = (torch.full((B, N, H, d), float("nan"), dtype=torch.float32, device=DEV) for _ in range(2))
+    rstd = torch.full((B, N, H), float("nan"), dtype=torch.float32, device=DEV)
+    ws = la.alloc_workspace(la.LA_OP_FWD, shape, DEV)
+    la.la_fwd_gated(shape, tm(q), tm(k), tm(v), tm(u), lam, y, o, rstd, None, None, ws)
+    torch.cuda.synchronize()
+    la.device_status()
+    assert_close(y.permute(0, 2, 1, 3), ref_y, TOL_BF16, "y")
+    assert_close(o.permute(0, 2, 1, 3), ref_o, TOL_BF16, "o")
+    r = rstd.permute(0, 2, 1).double().cpu().numpy()
+    assert np.max(np.abs(r - ref_rstd) / ref_rstd) <= 1e-3

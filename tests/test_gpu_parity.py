@@ -618,3 +618,53 @@ def test_decode_several_tokens_per_call(T, d):
     ref_o, ref_kv = orc.fwd_rec(q, k, v, lam.double().numpy(), kv_in=kv0.double().numpy(), want_state=True)
     assert_close(o_multi, ref_o, 1e-5, "o")
     assert_close(kv_multi, ref_kv, 1e-5, "state")
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("d", [64, 128])
+def test_token_major_layout(d, path):
+    """LA_LAYOUT_BNHD: the same tensors stored [B,N,H,d] (heads of a token adjacent) give the same results."""
+    if not path_ok(path, d, torch.bfloat16):
+        pytest.skip("tensor-core kernels do not cover this shape")
+    B, H, N = 2, 3, 777
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=71)
+    lam = torch.tensor([1.0, 0.96, 0.4])
+    kv_in = inputs.make_state(B, H, d, d, seed=72)
+    gko = inputs.make_state(B, H, d, d, seed=73)
+    ref = oracle_all(q, k, v, do, lam, kv_in.double().numpy(), gko.double().numpy())
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(DEV)      # [B,H,N,d] -> [B,N,H,d]
+    back = lambda x: x.permute(0, 2, 1, 3)
+    qg, kg, vg, dog = tm(q), tm(k), tm(v), tm(do)
+    kin, gk = to_dev(kv_in, gko)
+    for seg_len in (0, 256):
+        shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, seg_len, path, layout=la.LA_LAYOUT_BNHD)
+        o, dq, dk, dv = (torch.full((B, N, H, d), float("nan"), dtype=torch.float32, device=DEV) for _ in range(4))
+        kv_out, gin = (torch.empty((B, H, d, d), dtype=torch.float32, device=DEV) for _ in range(2))
+        ws_f = la.alloc_workspace(la.LA_OP_FWD, shape, DEV)
+        ws_b = la.alloc_workspace(la.LA_OP_BWD, shape, DEV)
+        la.la_fwd(shape, qg, kg, vg, lam, o, kin, kv_out, ws_f)
+        la.la_bwd(shape, qg, kg, vg, dog, lam, dq, dk, dv, kin, gk, gin, ws_b, fwd_workspace=ws_f)
+        torch.cuda.synchronize()
+        la.device_status()
+        compare_all((back(o), kv_out, back(dq), back(dk), back(dv), gin), ref,
+                    TOL_BF16 if path == la.LA_PATH_TENSOR else 1e-4)
+
+
+def test_token_major_layout_decode_steps():
+    B, H, T, d = 2, 4, 6, 128
+    lam = torch.tensor([1.0, 0.9, 0.5, 0.1])
+    gen = torch.Generator("cpu")
+    gen.manual_seed(74)
+    q = inputs.draw((B, H, T, d), gen, "silu", torch.bfloat16)
+    k = inputs.draw((B, H, T, d), gen, "silu", torch.bfloat16)
+    v = inputs.draw((B, H, T, d), gen, "normal", torch.bfloat16)
+    kv0 = inputs.make_state(B, H, d, d, seed=75)
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(DEV)
+    kv = kv0.to(DEV)
+    o = torch.empty((B, T, H, d), dtype=torch.float32, device=DEV)
+    shape = la.make_shape(B, H, T, d, d, torch.bfloat16, torch.float32, layout=la.LA_LAYOUT_BNHD)
+    la.la_decode_steps(shape, tm(q), tm(k), tm(v), lam, kv, o)
+    torch.cuda.synchronize()
+    ref_o, ref_kv = orc.fwd_rec(q, k, v, lam.double().numpy(), kv_in=kv0.double().numpy(), want_state=True)
+    assert_close(o.permute(0, 2, 1, 3), ref_o, 1e-5, "o")
+    assert_close(kv, ref_kv, 1e-5, "state")
