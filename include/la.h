@@ -201,6 +201,25 @@ la_status la_decode_step(const la_shape* shape, const void* q, const void* k, co
                          const float* lambda_host, float* kv, void* o, void* stream);
 
 /*
+ * Packed batches of sequences of different lengths (the serving-side form of Algorithm 2: every sequence has its
+ * own state).  The token tensors are [T, H, d] with the num_seqs sequences one after the other: shape->B = 1,
+ * shape->N = T, shape->layout = LA_LAYOUT_BNHD; cu_seqlens_host (HOST memory, num_seqs + 1 ints, cu[0] = 0,
+ * cu[num_seqs] = T, strictly increasing) gives the first token of each sequence.  Sequence i runs
+ * from the state kv_in[i] (or zero) and leaves kv_out[i]; kv_in, kv_out, grad_kv_out, grad_kv_in are
+ * [num_seqs, H, d, e] fp32 or NULL.  Results are those of la_fwd / la_bwd on each sequence alone.
+ * This version enqueues one la_fwd / la_bwd per sequence on `stream` (3 and 8 launches each), which suits a
+ * few long sequences; the workspace is shared: la_varlen_workspace_bytes gives the largest need of any sequence.
+ */
+size_t la_varlen_workspace_bytes(int op, const la_shape* shape, const int* cu_seqlens_host, int num_seqs);
+la_status la_fwd_varlen(const la_shape* shape, const void* q, const void* k, const void* v, const float* lambda_host,
+                        void* o, const int* cu_seqlens_host, int num_seqs, const float* kv_in, float* kv_out,
+                        void* workspace, size_t workspace_bytes, void* stream);
+la_status la_bwd_varlen(const la_shape* shape, const void* q, const void* k, const void* v, const void* d_o,
+                        const float* lambda_host, void* dq, void* dk, void* dv, const int* cu_seqlens_host, int num_seqs,
+                        const float* kv_in, const float* grad_kv_out, float* grad_kv_in, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/*
  * Several recurrent decode steps in one call (Algorithm 2 iterated over shape->N >= 1 consecutive tokens): for
  * t = 0 .. N-1 in order,  kv <- lambda_h kv + k_t v_t^T,  o_t <- kv^T q_t.
  *   q, k [B,H,N,d], v [B,H,N,e] in in_dtype; o [B,H,N,e] in out_dtype; kv [B,H,d,e] fp32, updated IN PLACE once.

@@ -26,7 +26,8 @@ LA_LAYOUT_BHND, LA_LAYOUT_BNHD = 0, 1
 EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_decode_step",
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
            "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
-           "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd", "la_decode_steps")
+           "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd", "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
+           "la_bwd_varlen")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate")
 
@@ -78,6 +79,13 @@ def load():
         lib.la_bwd_reuse.restype = I
         lib.la_decode_step.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_step.restype = I
+        ip = ctypes.POINTER(ctypes.c_int)
+        lib.la_varlen_workspace_bytes.argtypes = [I, sp, ip, I]
+        lib.la_varlen_workspace_bytes.restype = sz
+        lib.la_fwd_varlen.argtypes = [sp, vp, vp, vp, fp, vp, ip, I, vp, vp, vp, sz, vp]
+        lib.la_fwd_varlen.restype = I
+        lib.la_bwd_varlen.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, ip, I, vp, vp, vp, vp, sz, vp]
+        lib.la_bwd_varlen.restype = I
         lib.la_decode_steps.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_steps.restype = I
         lib.la_host_arena_bytes.argtypes = [sp]
@@ -257,7 +265,42 @@ def la_decode_steps(shape: LaShape, q, k, v, lam, kv, o, stream=None):
     rc = load().la_decode_steps(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(kv),
                                 _ptr(o), _stream(stream))
     if rc != 0:
-        raise LaError(rc, "la_decode_steps")
+        raise LaError(rc, "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
+           "la_bwd_varlen")
+
+
+def _cu(cu_seqlens):
+    vals = [int(x) for x in cu_seqlens]
+    return (ctypes.c_int * len(vals))(*vals), len(vals) - 1
+
+
+def varlen_workspace_bytes(op: int, shape: LaShape, cu_seqlens) -> int:
+    cu, S = _cu(cu_seqlens)
+    n = load().la_varlen_workspace_bytes(op, ctypes.byref(shape), cu, S)
+    if n == ctypes.c_size_t(-1).value:
+        raise LaError(2, "la_varlen_workspace_bytes")
+    return int(n)
+
+
+def la_fwd_varlen(shape: LaShape, q, k, v, lam, o, cu_seqlens, kv_in=None, kv_out=None, workspace=None, stream=None):
+    """Packed [T,H,d] tensors (shape: B=1, N=T, layout BNHD); cu_seqlens: host ints, first token of each sequence."""
+    cu, S = _cu(cu_seqlens)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_fwd_varlen(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(o), cu, S, _ptr(kv_in),
+                              _ptr(kv_out), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_fwd_varlen")
+
+
+def la_bwd_varlen(shape: LaShape, q, k, v, do, lam, dq, dk, dv, cu_seqlens, kv_in=None, grad_kv_out=None,
+                  grad_kv_in=None, workspace=None, stream=None):
+    cu, S = _cu(cu_seqlens)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_bwd_varlen(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(do), _lam(lam), _ptr(dq), _ptr(dk),
+                              _ptr(dv), cu, S, _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in), _ptr(workspace),
+                              ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_bwd_varlen")
 
 
 def host_arena_bytes(shape: LaShape) -> int:

@@ -615,6 +615,84 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
   return LA_OK;
 }
 
+// ---- packed batches of sequences of different lengths -------------------------------------------------------
+namespace {
+// Checks the packed description and returns, through `sub`, the shape of one sequence (N filled in per sequence).
+la_status varlen_check(const la_shape* shape, const int* cu, int S, la_shape* sub) {
+  la_status st = check_shape(shape, true);
+  if (st != LA_OK) return st;
+  if (!cu || S < 1) return LA_ERR_INVALID_ARG;
+  if (shape->B != 1 || shape->layout != LA_LAYOUT_BNHD) return LA_ERR_UNSUPPORTED;
+  if (cu[0] != 0 || cu[S] != shape->N) return LA_ERR_INVALID_ARG;
+  for (int i = 0; i < S; ++i)
+    if (cu[i + 1] <= cu[i]) return LA_ERR_INVALID_ARG;  // empty sequences are not allowed
+  *sub = *shape;
+  return LA_OK;
+}
+size_t esize(int dt) { return dt == LA_BF16 ? 2 : 4; }
+}  // namespace
+
+size_t la_varlen_workspace_bytes(int op, const la_shape* shape, const int* cu_seqlens_host, int num_seqs) {
+  la_shape sub;
+  if (op != LA_OP_FWD && op != LA_OP_BWD) return (size_t)-1;
+  if (varlen_check(shape, cu_seqlens_host, num_seqs, &sub) != LA_OK) return (size_t)-1;
+  size_t most = 0;
+  for (int i = 0; i < num_seqs; ++i) {
+    sub.N = cu_seqlens_host[i + 1] - cu_seqlens_host[i];
+    const size_t w = la_workspace_bytes(op, &sub);
+    if (w == (size_t)-1) return (size_t)-1;
+    if (w > most) most = w;
+  }
+  return most;
+}
+
+la_status la_fwd_varlen(const la_shape* shape, const void* q, const void* k, const void* v, const float* lambda_host,
+                        void* o, const int* cu_seqlens_host, int num_seqs, const float* kv_in, float* kv_out,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  la_shape sub;
+  la_status st = varlen_check(shape, cu_seqlens_host, num_seqs, &sub);
+  if (st != LA_OK) return st;
+  if (!q || !k || !v || !o) return LA_ERR_INVALID_ARG;
+  const size_t row_in = (size_t)shape->H * shape->d * esize(shape->in_dtype);
+  const size_t row_out = (size_t)shape->H * shape->e * esize(shape->out_dtype);
+  const size_t state = (size_t)shape->H * shape->d * shape->e;
+  for (int i = 0; i < num_seqs; ++i) {
+    const size_t t0 = (size_t)cu_seqlens_host[i];
+    sub.N = cu_seqlens_host[i + 1] - cu_seqlens_host[i];
+    st = la_fwd(&sub, static_cast<const char*>(q) + t0 * row_in, static_cast<const char*>(k) + t0 * row_in,
+                static_cast<const char*>(v) + t0 * row_in, lambda_host, static_cast<char*>(o) + t0 * row_out,
+                kv_in ? kv_in + i * state : nullptr, kv_out ? kv_out + i * state : nullptr, workspace, workspace_bytes,
+                stream);
+    if (st != LA_OK) return st;
+  }
+  return LA_OK;
+}
+
+la_status la_bwd_varlen(const la_shape* shape, const void* q, const void* k, const void* v, const void* d_o,
+                        const float* lambda_host, void* dq, void* dk, void* dv, const int* cu_seqlens_host, int num_seqs,
+                        const float* kv_in, const float* grad_kv_out, float* grad_kv_in, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+  la_shape sub;
+  la_status st = varlen_check(shape, cu_seqlens_host, num_seqs, &sub);
+  if (st != LA_OK) return st;
+  if (!q || !k || !v || !d_o || !dq || !dk || !dv) return LA_ERR_INVALID_ARG;
+  const size_t row_in = (size_t)shape->H * shape->d * esize(shape->in_dtype);
+  const size_t row_out = (size_t)shape->H * shape->e * esize(shape->out_dtype);
+  const size_t state = (size_t)shape->H * shape->d * shape->e;
+  for (int i = 0; i < num_seqs; ++i) {
+    const size_t t0 = (size_t)cu_seqlens_host[i];
+    sub.N = cu_seqlens_host[i + 1] - cu_seqlens_host[i];
+    st = la_bwd(&sub, static_cast<const char*>(q) + t0 * row_in, static_cast<const char*>(k) + t0 * row_in,
+                static_cast<const char*>(v) + t0 * row_in, static_cast<const char*>(d_o) + t0 * row_in, lambda_host,
+                static_cast<char*>(dq) + t0 * row_out, static_cast<char*>(dk) + t0 * row_out,
+                static_cast<char*>(dv) + t0 * row_out, kv_in ? kv_in + i * state : nullptr,
+                grad_kv_out ? grad_kv_out + i * state : nullptr, grad_kv_in ? grad_kv_in + i * state : nullptr, workspace,
+                workspace_bytes, stream);
+    if (st != LA_OK) return st;
+  }
+  return LA_OK;
+}
+
 la_status la_selftest_bounded_wait(unsigned long long budget_clocks, void* stream) {
   if (budget_clocks == 0 || budget_clocks > 2000000000ull) return LA_ERR_INVALID_ARG;
   const la_status dev = check_device();

@@ -668,3 +668,39 @@ def test_token_major_layout_decode_steps():
     ref_o, ref_kv = orc.fwd_rec(q, k, v, lam.double().numpy(), kv_in=kv0.double().numpy(), want_state=True)
     assert_close(o.permute(0, 2, 1, 3), ref_o, 1e-5, "o")
     assert_close(kv, ref_kv, 1e-5, "state")
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_packed_sequences_of_different_lengths(d):
+    """la_fwd_varlen / la_bwd_varlen: sequences packed one after the other in [T,H,d] tensors, each with its own
+    state; every sequence against the oracle run on that sequence alone."""
+    H = 3
+    lens = [1, 130, 700, 257, 64]
+    cu = [0]
+    for n in lens:
+        cu.append(cu[-1] + n)
+    T, S = cu[-1], len(lens)
+    lam = torch.tensor([1.0, 0.95, 0.3])
+    q, k, v, do = inputs.make_qkvdo(1, H, T, d, d, seed=91)           # [1,H,T,d]
+    kv_in = inputs.make_state(S, H, d, d, seed=92)
+    gko = inputs.make_state(S, H, d, d, seed=93)
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(DEV)           # packed [1,T,H,d]
+    qg, kg, vg, dog = tm(q), tm(k), tm(v), tm(do)
+    shape = la.make_shape(1, H, T, d, d, torch.bfloat16, torch.float32, 256, layout=la.LA_LAYOUT_BNHD)
+    o, dq, dk, dv = (torch.full((1, T, H, d), float("nan"), dtype=torch.float32, device=DEV) for _ in range(4))
+    kv_out, gin = (torch.empty((S, H, d, d), dtype=torch.float32, device=DEV) for _ in range(2))
+    ws_f = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_FWD, shape, cu), 256), dtype=torch.uint8, device=DEV)
+    ws_b = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_BWD, shape, cu), 256), dtype=torch.uint8, device=DEV)
+    la.la_fwd_varlen(shape, qg, kg, vg, lam, o, cu, kv_in.to(DEV), kv_out, ws_f)
+    la.la_bwd_varlen(shape, qg, kg, vg, dog, lam, dq, dk, dv, cu, kv_in.to(DEV), gko.to(DEV), gin, ws_b)
+    torch.cuda.synchronize()
+    la.device_status()
+    back = lambda x, a, b: x[:, a:b].permute(0, 2, 1, 3)
+    for i in range(S):
+        a, b = cu[i], cu[i + 1]
+        ref = oracle_all(q[:, :, a:b], k[:, :, a:b], v[:, :, a:b], do[:, :, a:b], lam,
+                         kv_in[i:i + 1].double().numpy(), gko[i:i + 1].double().numpy())
+        got = (back(o, a, b), kv_out[i:i + 1], back(dq, a, b), back(dk, a, b), back(dv, a, b), gin[i:i + 1])
+        compare_all(got, ref, TOL_BF16)
+    with pytest.raises(la.LaError):     # the description must cover the tensor exactly
+        la.la_fwd_varlen(shape, qg, kg, vg, lam, o, cu[:-1] + [T - 1], None, None, ws_f)
