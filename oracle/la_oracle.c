@@ -39,7 +39,12 @@
  *   - SimpleRMSNorm is applied to each head's e output values of a token (the
  *     model-parallel form of Eq. 3 normalises each rank's heads on their own);
  *     Eq. 8 has no epsilon, so a row with ||o||_2 = 0 is given y = 0 and zero
- *     gradients.
+ *     gradients;
+ *   - Eq. 1's rotation (LRPE-d): theta is one learnable angle per head and per
+ *     feature, the score is the real part of the complex expression,
+ *       a_ts = lambda^(t-s) sum_i q_t[i] k_s[i] cos(theta[h][i] (t - s)),  s <= t
+ *     (the paper prints a bare theta; the cited LRPE work uses one angle per
+ *     feature, and a single angle is the special case of equal entries).
  *
  * Every routine is pinned by tests that do not call it twice: closed forms,
  * a hand-worked example, numpy prefix sums for lambda = 1, brute force on tiny
@@ -419,4 +424,120 @@ int orc_norm_gate_bwd(const double* o, const float* u, const float* dy, long row
     }
   }
   return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* LRPE-d (Eq. 1): decay and a learnable rotation of the relative position.    */
+/*   a_ts = lambda^(t-s) sum_i q_t[i] k_s[i] cos(theta_i (t-s))   (s <= t)     */
+/*   o_t  = sum_{s<=t} a_ts v_s                                                */
+/* theta [H, d] fp64.  The N x N matrix is materialised as in orc_fwd_quad.    */
+/* ------------------------------------------------------------------------- */
+int orc_lrpe_fwd_quad(const float* q, const float* k, const float* v, const double* lambda,
+                      const double* theta, int B, int H, int N, int d, int e, double* o) {
+  if (B < 0 || H < 0 || N < 0 || d < 1 || e < 1) return ORC_ERR;
+  if ((double)N * (double)N > 2.0e8) return ORC_ERR;
+  const long BH = (long)B * H;
+  int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < BH; ++bh) {
+    const double lam = lambda[bh % H];
+    const double* th = theta + (size_t)(bh % H) * d;
+    double* A = (double*)malloc(sizeof(double) * (size_t)N * N);
+    if (!A) { failed = 1; continue; }
+    for (long t = 0; t < N; ++t)
+      for (long s = 0; s < N; ++s) {
+        double a = 0.0;
+        if (t >= s) {
+          for (int i = 0; i < d; ++i)
+            a += (double)q[(bh * N + t) * d + i] * (double)k[(bh * N + s) * d + i] * cos(th[i] * (double)(t - s));
+          a *= mask_entry(lam, t - s);
+        }
+        A[t * N + s] = a;
+      }
+    for (long t = 0; t < N; ++t)
+      for (int j = 0; j < e; ++j) {
+        double acc = 0.0;
+        for (long s = 0; s < N; ++s) acc += A[t * N + s] * (double)v[(bh * N + s) * e + j];
+        o[(bh * N + t) * e + j] = acc;
+      }
+    free(A);
+  }
+  return failed ? ORC_ERR : ORC_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Gradients of L = <O, dO> for LRPE-d.  With dA_ts = lambda^(t-s) do_t.v_s:   */
+/*   dq_t[i]   =  sum_{s<=t} dA_ts k_s[i] cos(theta_i (t-s))                   */
+/*   dk_s[i]   =  sum_{t>=s} dA_ts q_t[i] cos(theta_i (t-s))                   */
+/*   dv_s      =  sum_{t>=s} a_ts do_t                                         */
+/*   dtheta_i  = -sum_{b} sum_{s<=t} dA_ts q_t[i] k_s[i] (t-s) sin(theta_i (t-s))   (theta is shared by the batch) */
+/* dtheta [H, d].                                                              */
+/* ------------------------------------------------------------------------- */
+int orc_lrpe_bwd_quad(const float* q, const float* k, const float* v, const float* d_o,
+                      const double* lambda, const double* theta, int B, int H, int N, int d, int e,
+                      double* dq, double* dk, double* dv, double* dtheta) {
+  if (B < 0 || H < 0 || N < 0 || d < 1 || e < 1) return ORC_ERR;
+  if ((double)N * (double)N > 1.0e8) return ORC_ERR;
+  const long BH = (long)B * H;
+  int failed = 0;
+  double* dth_part = (double*)calloc((size_t)(BH > 0 ? BH : 1) * d, sizeof(double)); /* one row per (b,h) */
+  if (!dth_part) return ORC_ERR;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long bh = 0; bh < BH; ++bh) {
+    const double lam = lambda[bh % H];
+    const double* th = theta + (size_t)(bh % H) * d;
+    double* A = (double*)malloc(sizeof(double) * (size_t)N * N);
+    double* dA = (double*)malloc(sizeof(double) * (size_t)N * N);
+    if (!A || !dA) { failed = 1; free(A); free(dA); continue; }
+    for (long t = 0; t < N; ++t)
+      for (long s = 0; s < N; ++s) {
+        double a = 0.0, da = 0.0;
+        if (t >= s) {
+          const double m = mask_entry(lam, t - s);
+          for (int i = 0; i < d; ++i)
+            a += (double)q[(bh * N + t) * d + i] * (double)k[(bh * N + s) * d + i] * cos(th[i] * (double)(t - s));
+          for (int j = 0; j < e; ++j)
+            da += (double)d_o[(bh * N + t) * e + j] * (double)v[(bh * N + s) * e + j];
+          a *= m;
+          da *= m;
+        }
+        A[t * N + s] = a;
+        dA[t * N + s] = da;
+      }
+    for (long t = 0; t < N; ++t)
+      for (int i = 0; i < d; ++i) {
+        double acc = 0.0;
+        for (long s = 0; s <= t; ++s)
+          acc += dA[t * N + s] * (double)k[(bh * N + s) * d + i] * cos(th[i] * (double)(t - s));
+        dq[(bh * N + t) * d + i] = acc;
+      }
+    for (long s = 0; s < N; ++s)
+      for (int i = 0; i < d; ++i) {
+        double acc = 0.0;
+        for (long t = s; t < N; ++t)
+          acc += dA[t * N + s] * (double)q[(bh * N + t) * d + i] * cos(th[i] * (double)(t - s));
+        dk[(bh * N + s) * d + i] = acc;
+      }
+    for (long s = 0; s < N; ++s)
+      for (int j = 0; j < e; ++j) {
+        double acc = 0.0;
+        for (long t = 0; t < N; ++t) acc += A[t * N + s] * (double)d_o[(bh * N + t) * e + j];
+        dv[(bh * N + s) * e + j] = acc;
+      }
+    for (int i = 0; i < d; ++i) {
+      double acc = 0.0;
+      for (long t = 0; t < N; ++t)
+        for (long s = 0; s <= t; ++s)
+          acc -= dA[t * N + s] * (double)q[(bh * N + t) * d + i] * (double)k[(bh * N + s) * d + i] *
+                 (double)(t - s) * sin(th[i] * (double)(t - s));
+      dth_part[bh * d + i] = acc;
+    }
+    free(A);
+    free(dA);
+  }
+  for (long hi = 0; hi < (long)H * d; ++hi) dtheta[hi] = 0.0;
+  for (long bh = 0; bh < BH; ++bh)
+    for (int i = 0; i < d; ++i) dtheta[(bh % H) * d + i] += dth_part[bh * d + i];
+  free(dth_part);
+  return failed ? ORC_ERR : ORC_OK;
 }

@@ -50,6 +50,8 @@ def _load():
         lib.orc_rows.argtypes = [I, fp, fp, fp, fp, dp, I, I, I, I, I, I, ip, ip, dp]
         lib.orc_decode_step.argtypes = [fp, fp, fp, dp, dp, I, I, I, I, dp]
         lib.orc_fwd_origin.argtypes = [fp, fp, fp, dp, I, I, I, I, I, dp]
+        lib.orc_lrpe_fwd_quad.argtypes = [fp, fp, fp, dp, dp, I, I, I, I, I, dp]
+        lib.orc_lrpe_bwd_quad.argtypes = [fp, fp, fp, fp, dp, dp, I, I, I, I, I, dp, dp, dp, dp]
         lib.orc_norm_gate_fwd.argtypes = [dp, fp, ctypes.c_long, I, dp, dp]
         lib.orc_norm_gate_bwd.argtypes = [dp, fp, fp, ctypes.c_long, I, dp, dp]
         for name in ("orc_fwd_rec", "orc_bwd_rec", "orc_fwd_quad", "orc_bwd_quad", "orc_rows",
@@ -228,3 +230,32 @@ def norm_gate_bwd(o, u, dy):
     _check(_load().orc_norm_gate_bwd(_p(o, D), _p(u, F), _p(dy, F), ctypes.c_long(rows), e, _p(d_o, D), _p(d_u, D)),
            "orc_norm_gate_bwd")
     return d_o, d_u
+
+
+def lrpe_fwd_quad(q, k, v, lam, theta):
+    """LRPE-d (Eq. 1): o_t = sum_{s<=t} lambda^(t-s) sum_i q_t[i] k_s[i] cos(theta[h,i] (t-s)) v_s.  theta [H, d]."""
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    B, H, N, d, e = _dims(q, v)
+    lam, theta = _f64(lam), _f64(theta)
+    assert theta.shape == (H, d)
+    o = np.empty((B, H, N, e), np.float64)
+    D, F = ctypes.c_double, ctypes.c_float
+    _check(_load().orc_lrpe_fwd_quad(_p(q, F), _p(k, F), _p(v, F), _p(lam, D), _p(theta, D), B, H, N, d, e, _p(o, D)),
+           "orc_lrpe_fwd_quad")
+    return o
+
+
+def lrpe_bwd_quad(q, k, v, do, lam, theta):
+    """Gradients of <O, dO> for LRPE-d with respect to q, k, v and theta ([H, d], summed over the batch)."""
+    q, k, v, do = _f32(q), _f32(k), _f32(v), _f32(do)
+    B, H, N, d, e = _dims(q, v)
+    lam, theta = _f64(lam), _f64(theta)
+    assert theta.shape == (H, d)
+    dq = np.empty((B, H, N, d), np.float64)
+    dk = np.empty((B, H, N, d), np.float64)
+    dv = np.empty((B, H, N, e), np.float64)
+    dth = np.empty((H, d), np.float64)
+    D, F = ctypes.c_double, ctypes.c_float
+    _check(_load().orc_lrpe_bwd_quad(_p(q, F), _p(k, F), _p(v, F), _p(do, F), _p(lam, D), _p(theta, D), B, H, N, d, e,
+                                     _p(dq, D), _p(dk, D), _p(dv, D), _p(dth, D)), "orc_lrpe_bwd_quad")
+    return dq, dk, dv, dth

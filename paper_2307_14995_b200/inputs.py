@@ -98,6 +98,18 @@ def make_state(B: int, H: int, d: int, e: int, *, seed: int = 1, scale: float = 
     return (torch.randn((B, H, d, e), generator=gen, dtype=torch.float32) * scale).contiguous()
 
 
+def make_theta(H: int, d: int, *, seed: int = 2, base: float = 10000.0, jitter: float = 0.1) -> torch.Tensor:
+    """Rotation angles for LRPE-d (Eq. 1), fp32 [H, d]: geometrically spaced frequencies base^(-i/d) (the usual
+    initialisation of rotary-style encodings) times a seeded log-normal factor per (head, feature), standing in for
+    values a short stretch of training would have moved them to."""
+    gen = torch.Generator("cpu")
+    gen.manual_seed(seed)
+    i = torch.arange(d, dtype=torch.float64)
+    freq = torch.pow(torch.tensor(base, dtype=torch.float64), -i / d)
+    z = torch.randn((H, d), generator=gen, dtype=torch.float32).double()
+    return (freq[None, :] * torch.exp(jitter * z)).float().contiguous()
+
+
 def make_workload(name: str, *, B: Optional[int] = None, H: Optional[int] = None, N: Optional[int] = None):
     """Inputs of a named workload (optionally with reduced B/H/N for sampled checks).
 

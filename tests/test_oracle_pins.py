@@ -429,3 +429,123 @@ def test_norm_gate_invariants_and_finite_differences():
     # a zero row is given y = 0 and zero gradients (Eq. 8 has no epsilon)
     z = np.zeros((1, e))
     assert np.all(orc.norm_gate_fwd(z, u[:1]) == 0) and np.all(orc.norm_gate_bwd(z, u[:1], dy[:1])[0] == 0)
+
+
+# --- LRPE-d (Eq. 1): decay and rotation of the relative position ---------------------------------------------
+def lrpe_features(x, theta, pos0=0):
+    """[x cos(theta t), x sin(theta t)] along the feature axis: the split of Eq. 1's rotation into a factor that
+    depends on the query position only and one that depends on the key position only."""
+    x = np.asarray(x, np.float64)
+    N = x.shape[2]
+    ang = np.asarray(theta, np.float64)[None, :, None, :] * (pos0 + np.arange(N, dtype=np.float64))[None, None, :, None]
+    return np.concatenate([x * np.cos(ang), x * np.sin(ang)], axis=-1)
+
+
+def test_lrpe_hand_worked_two_tokens():
+    g = json.load(open(os.path.join(HERE, "golden", "lrpe_example.json")))
+    sh = (1, 1, 2, 2)
+    q, k, v, do = (np.array(g[n], np.float32).reshape(sh) for n in ("q", "k", "v", "dO"))
+    lam, th = np.array([g["lambda"]]), np.array([g["theta"]])
+    o = orc.lrpe_fwd_quad(q, k, v, lam, th)
+    np.testing.assert_allclose(o.ravel(), np.array(g["o"]), rtol=0, atol=1e-14)
+    dq, dk, dv, dth = orc.lrpe_bwd_quad(q, k, v, do, lam, th)
+    for got, name in ((dq, "dq"), (dk, "dk"), (dv, "dv"), (dth, "dtheta")):
+        np.testing.assert_allclose(got.ravel(), np.array(g[name]), rtol=0, atol=1e-14, err_msg=name)
+
+
+def test_lrpe_zero_angle_is_the_plain_operator():
+    q, k, v, do = rand_inputs(2, 3, 40, 8, 6, seed=5)
+    lam = np.array([1.0, 0.9, 0.4])
+    th = np.zeros((3, 8))
+    np.testing.assert_allclose(orc.lrpe_fwd_quad(q, k, v, lam, th), orc.fwd_quad(q, k, v, lam), rtol=0, atol=1e-13)
+    got = orc.lrpe_bwd_quad(q, k, v, do, lam, th)
+    ref = orc.bwd_quad(q, k, v, do, lam)
+    for a, b in zip(got[:3], ref):
+        np.testing.assert_allclose(a, b, rtol=0, atol=1e-12)
+    assert np.all(got[3] == 0.0)        # sin(0) = 0: no first-order dependence on theta at theta = 0
+
+
+def test_lrpe_is_the_real_part_of_the_complex_form():
+    """Eq. 1 as printed: a_ts = q_t^T k_s lambda^(t-s) exp(i theta (t-s)), evaluated with complex numbers."""
+    B, H, N, d, e = 1, 2, 33, 6, 5
+    q, k, v, _ = rand_inputs(B, H, N, d, e, seed=6)
+    q, k, v = (np.asarray(x, np.float64) for x in (q, k, v))
+    lam = np.array([0.97, 0.6])
+    th = inputs.make_theta(H, d, seed=3).double().numpy() * 50.0       # angles large enough to wrap within 33 tokens
+    t = np.arange(N)
+    rot = np.exp(1j * th[None, :, None, :] * t[None, None, :, None])    # [1,H,N,d]
+    scores = np.einsum("bhti,bhsi->bhts", q * rot, np.conj(k * rot))
+    mask = np.tril(np.power(lam[:, None, None], (t[:, None] - t[None, :]).clip(min=0)[None]))
+    o_ref = np.einsum("bhts,bhsj->bhtj", (scores * mask[None]).real, v)
+    assert relerr(orc.lrpe_fwd_quad(q, k, v, lam, th), o_ref) < 1e-12
+
+
+@pytest.mark.parametrize("pos0", [0, 1000])
+def test_lrpe_separates_into_position_features(pos0):
+    """cos(a - b) = cos a cos b + sin a sin b: the plain operator on doubled features [x cos, x sin], evaluated at
+    absolute positions (any common offset), equals the relative-position definition, for outputs and for the
+    gradients with respect to v."""
+    B, H, N, d, e = 2, 2, 50, 4, 3
+    q, k, v, do = rand_inputs(B, H, N, d, e, seed=7)
+    lam = np.array([1.0, 0.8])
+    th = inputs.make_theta(H, d, seed=4).double().numpy() * 20.0
+    qf, kf = lrpe_features(q, th, pos0), lrpe_features(k, th, pos0)
+    o = orc.lrpe_fwd_quad(q, k, v, lam, th)
+    assert relerr(orc.fwd_quad(qf.astype(np.float32), kf.astype(np.float32), v, lam), o) < 1e-5   # fp32 containers
+    # in fp64 throughout (the recurrence takes fp32 containers, so use the einsum definition here)
+    t = np.arange(N)
+    mask = np.tril(np.power(lam[:, None, None], (t[:, None] - t[None, :]).clip(min=0)[None]))
+    o2 = np.einsum("bhts,bhsj->bhtj", np.einsum("bhti,bhsi->bhts", qf, kf) * mask[None], np.asarray(v, np.float64))
+    assert relerr(o2, o) < 1e-12
+    dv = orc.lrpe_bwd_quad(q, k, v, do, lam, th)[2]
+    dv2 = np.einsum("bhts,bhtj->bhsj", np.einsum("bhti,bhsi->bhts", qf, kf) * mask[None], np.asarray(do, np.float64))
+    assert relerr(dv2, dv) < 1e-12
+
+
+def test_lrpe_finite_differences():
+    B, H, N, d, e = 2, 2, 12, 3, 4
+    q, k, v, do = (np.asarray(x, np.float64) for x in rand_inputs(B, H, N, d, e, seed=8))
+    lam = np.array([0.95, 0.5])
+    th = np.array([[0.3, 1.1, 2.0], [0.05, 0.7, 1.6]])
+
+    def loss(q_, k_, v_, th_):
+        return float(np.sum(orc.lrpe_fwd_quad(q_, k_, v_, lam, th_) * do))
+
+    dq, dk, dv, dth = orc.lrpe_bwd_quad(q, k, v, do, lam, th)
+    rng = np.random.default_rng(0)
+    # inputs are carried in fp32 containers: perturb by values exactly representable there
+    h = 2.0 ** -10
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        for _ in range(6):
+            idx = tuple(rng.integers(0, n) for n in x.shape)
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += h
+            xm[idx] -= h
+            args_p = {"q": (xp, k, v), "k": (q, xp, v), "v": (q, k, xp)}[name]
+            args_m = {"q": (xm, k, v), "k": (q, xm, v), "v": (q, k, xm)}[name]
+            fd = (loss(*args_p, th) - loss(*args_m, th)) / (2 * h)      # exact: the loss is linear in each of q, k, v
+            assert abs(fd - g[idx]) < 1e-9 * (1 + abs(fd)), (name, idx)
+    for hh in range(H):
+        for i in range(d):
+            tp, tm = th.copy(), th.copy()
+            tp[hh, i] += 1e-5
+            tm[hh, i] -= 1e-5
+            fd = (loss(q, k, v, tp) - loss(q, k, v, tm)) / 2e-5
+            assert abs(fd - dth[hh, i]) < 1e-6 * (1 + abs(fd)), (hh, i)
+
+
+def test_lrpe_brute_force_loops():
+    B, H, N, d, e = 1, 2, 7, 2, 2
+    q, k, v, _ = (np.asarray(x, np.float64) for x in rand_inputs(B, H, N, d, e, seed=9))
+    lam = [0.9, 0.3]
+    th = [[0.4, 1.3], [2.2, 0.01]]
+    o = np.zeros((B, H, N, e))
+    for h in range(H):
+        for t in range(N):
+            for s in range(t + 1):
+                a = 0.0
+                for i in range(d):
+                    a += q[0, h, t, i] * k[0, h, s, i] * np.cos(th[h][i] * (t - s))
+                for j in range(e):
+                    o[0, h, t, j] += lam[h] ** (t - s) * a * v[0, h, s, j]
+    np.testing.assert_allclose(orc.lrpe_fwd_quad(q, k, v, np.array(lam), np.array(th)), o, rtol=0, atol=1e-13)
