@@ -373,6 +373,23 @@ def run_ours(args):
                  "gate_bwd_gbs": th * (eb * w.d + 3 * 2 * w.d + eb * w.d) / (gbwd_ms * 1e-3) / 1e9}
         del ug, yg, dyg, dog
 
+    # ---- LRPE-d (Eq. 1), the first layer's variant: feature doubling around two runs of the operator ----
+    lrpe = None
+    if train_steps and args.only == "all":
+        theta = inputs.make_theta(w.H, w.d, seed=2).to(dev)
+        dth = torch.empty((w.H, w.d), dtype=torch.float32, device=dev)
+        wl_f = torch.empty(la.lrpe_workspace_bytes(la.LA_OP_FWD, shape), dtype=torch.uint8, device=dev)
+        lf_ms, lf_l = time_loop(lambda: la.la_lrpe_fwd(shape, q, k, v, theta, lam, o, 0, None, None, wl_f, stream), n=5)
+        wl_b = torch.empty(la.lrpe_workspace_bytes(la.LA_OP_BWD, shape), dtype=torch.uint8, device=dev)
+        lb_ms, lb_l = time_loop(lambda: la.la_lrpe_bwd(shape, q, k, v, do, theta, lam, dq, dk, dv, dth, 0, None, None, None,
+                                                       wl_b, stream), n=5)
+        lrpe = {"what": "la_lrpe_fwd + la_lrpe_bwd at the same shape (rotation of Eq. 1 as position features, doubled "
+                        "feature dimension = two runs of the operator plus element-wise kernels)",
+                "fwd_ms": lf_ms, "bwd_ms": lb_ms, "fwd_launches": lf_l, "bwd_launches": lb_l,
+                "ratio_to_plain_step": (lf_ms + lb_ms) / ms_step,
+                "workspace_bytes": {"fwd": wl_f.numel(), "bwd": wl_b.numel()}}
+        del wl_f, wl_b, theta, dth
+
     # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
     dw = inputs.WORKLOADS["decode"]
     gen = torch.Generator(dev)
@@ -531,7 +548,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / prof_steps for kname, (ms, _) in prof.items()},
             "kernel_launches_per_step": {kname: c / prof_steps for kname, (_, c) in prof.items()},
-            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated,
+            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe,
             "roofline": {"scope": "ONE kernel, the dominant one; the whole-step figure the target is stated on is step_roofline",
                          "kernel": "full-width block walk (tc_walk_full_kernel), single-job launches (O and dQ)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -201,6 +201,30 @@ la_status la_decode_step(const la_shape* shape, const void* q, const void* k, co
                          const float* lambda_host, float* kv, void* o, void* stream);
 
 /*
+ * LRPE-d (Eq. 1): decay times a learnable rotation of the relative position,
+ *   a_ts = lambda^(t-s) sum_i q_t[i] k_s[i] cos(theta[h][i] (t-s)),  s <= t;   o_t = sum_{s<=t} a_ts v_s
+ * (the real part of the printed complex form; one angle per head and feature).  The rotation splits into the
+ * position features [x cos(theta t), x sin(theta t)], i.e. a doubled feature dimension 2d, and the result is the
+ * sum of two runs of the decayed operator on the two halves, which is how these calls compute it.
+ *   theta        DEVICE, [H,d] fp32, 16-byte aligned;       d_theta  OUT, DEVICE, [H,d] fp32 (overwritten);
+ *   pos0         absolute position of the first token (>= 0; chunks of one sequence pass their offset);
+ *   kv_in, kv_out, grad_kv_out, grad_kv_in   [2,B,H,d,e] fp32 (cos half, then sin half) or NULL;
+ *   other arguments as in la_fwd / la_bwd; requires d == e.
+ * Workspace: la_lrpe_workspace_bytes(op, shape), 256-byte aligned: the four feature tensors, fp32 temporaries of
+ * the tensors' size (1-2 forward, 5-6 backward) and the inner calls' own workspace.
+ * d_theta is a position-weighted sum whose q and k parts cancel down to the relative-position result; with
+ * bf16 features its error grows with the absolute positions (see the tests for the bound that is checked).
+ */
+size_t la_lrpe_workspace_bytes(int op, const la_shape* shape);
+la_status la_lrpe_fwd(const la_shape* shape, const void* q, const void* k, const void* v, const float* theta,
+                      const float* lambda_host, long long pos0, void* o, const float* kv_in, float* kv_out,
+                      void* workspace, size_t workspace_bytes, void* stream);
+la_status la_lrpe_bwd(const la_shape* shape, const void* q, const void* k, const void* v, const void* d_o,
+                      const float* theta, const float* lambda_host, long long pos0, void* dq, void* dk, void* dv,
+                      float* d_theta, const float* kv_in, const float* grad_kv_out, float* grad_kv_in, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/*
  * Packed batches of sequences of different lengths (the serving-side form of Algorithm 2: every sequence has its
  * own state).  The token tensors are [T, H, d] with the num_seqs sequences one after the other: shape->B = 1,
  * shape->N = T, shape->layout = LA_LAYOUT_BNHD; cu_seqlens_host (HOST memory, num_seqs + 1 ints, cu[0] = 0,
@@ -336,7 +360,8 @@ unsigned long long la_launch_count(void);
 #define LA_KERNEL_DECODE 3  /* recurrent decode step           */
 #define LA_KERNEL_WALK_PAIR 4 /* the dV and dK walks of the backward pass in one launch */
 #define LA_KERNEL_GATE 5      /* stand-alone SRMSNorm-and-gate kernels (la_fwd_gated fallback, la_gate_bwd) */
-#define LA_NUM_KERNEL_KINDS 6
+#define LA_KERNEL_LRPE 6      /* element-wise kernels of la_lrpe_fwd / la_lrpe_bwd */
+#define LA_NUM_KERNEL_KINDS 7
 void la_profile_enable(int on);
 la_status la_profile_collect(double* ms, unsigned long long* launches);
 

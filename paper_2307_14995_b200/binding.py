@@ -27,9 +27,9 @@ EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_de
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
            "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
            "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd", "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
-           "la_bwd_varlen")
+           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
-KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate")
+KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate", "lrpe")
 
 
 class LaShape(ctypes.Structure):
@@ -86,6 +86,13 @@ def load():
         lib.la_fwd_varlen.restype = I
         lib.la_bwd_varlen.argtypes = [sp, vp, vp, vp, vp, fp, vp, vp, vp, ip, I, vp, vp, vp, vp, sz, vp]
         lib.la_bwd_varlen.restype = I
+        LL = ctypes.c_longlong
+        lib.la_lrpe_workspace_bytes.argtypes = [I, sp]
+        lib.la_lrpe_workspace_bytes.restype = sz
+        lib.la_lrpe_fwd.argtypes = [sp, vp, vp, vp, vp, fp, LL, vp, vp, vp, vp, sz, vp]
+        lib.la_lrpe_fwd.restype = I
+        lib.la_lrpe_bwd.argtypes = [sp, vp, vp, vp, vp, vp, fp, LL, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.la_lrpe_bwd.restype = I
         lib.la_decode_steps.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_steps.restype = I
         lib.la_host_arena_bytes.argtypes = [sp]
@@ -266,7 +273,7 @@ def la_decode_steps(shape: LaShape, q, k, v, lam, kv, o, stream=None):
                                 _ptr(o), _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
-           "la_bwd_varlen")
+           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd")
 
 
 def _cu(cu_seqlens):
@@ -300,7 +307,33 @@ def la_bwd_varlen(shape: LaShape, q, k, v, do, lam, dq, dk, dv, cu_seqlens, kv_i
                               _ptr(dv), cu, S, _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in), _ptr(workspace),
                               ws_bytes, _stream(stream))
     if rc != 0:
-        raise LaError(rc, "la_bwd_varlen")
+        raise LaError(rc, "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd")
+
+
+def lrpe_workspace_bytes(op: int, shape: LaShape) -> int:
+    n = load().la_lrpe_workspace_bytes(op, ctypes.byref(shape))
+    if n == ctypes.c_size_t(-1).value:
+        raise LaError(2, "la_lrpe_workspace_bytes")
+    return int(n)
+
+
+def la_lrpe_fwd(shape: LaShape, q, k, v, theta, lam, o, pos0=0, kv_in=None, kv_out=None, workspace=None, stream=None):
+    """LRPE-d forward (Eq. 1); theta: device fp32 [H,d]; states [2,B,H,d,e]."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_lrpe_fwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(theta), _lam(lam), int(pos0), _ptr(o),
+                            _ptr(kv_in), _ptr(kv_out), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_lrpe_fwd")
+
+
+def la_lrpe_bwd(shape: LaShape, q, k, v, do, theta, lam, dq, dk, dv, dtheta, pos0=0, kv_in=None, grad_kv_out=None,
+                grad_kv_in=None, workspace=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_lrpe_bwd(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(do), _ptr(theta), _lam(lam), int(pos0),
+                            _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dtheta), _ptr(kv_in), _ptr(grad_kv_out),
+                            _ptr(grad_kv_in), _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_lrpe_bwd")
 
 
 def host_arena_bytes(shape: LaShape) -> int:

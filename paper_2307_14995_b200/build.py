@@ -14,7 +14,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libla_b200.so")
-SOURCES = ["la_api.cu", "la_simt.cu", "la_decode.cu", "la_tc.cu", "la_noalloc.cu", "la_gate.cu"]
+SOURCES = ["la_api.cu", "la_simt.cu", "la_decode.cu", "la_tc.cu", "la_noalloc.cu", "la_gate.cu", "la_lrpe.cu"]
 HEADERS = ["la_common.cuh", os.path.join("..", "..", "include", "la.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC"]

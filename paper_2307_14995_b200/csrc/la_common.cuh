@@ -126,7 +126,7 @@ struct KernelTimer {
   cudaEvent_t start_;
   bool active_;
 };
-enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_WALK_PAIR = 4, K_GATE = 5, K_NUM = 6 };
+enum { K_PREPASS = 0, K_SCAN = 1, K_WALK = 2, K_DECODE = 3, K_WALK_PAIR = 4, K_GATE = 5, K_LRPE = 6, K_NUM = 7 };
 
 // ---- small device helpers --------------------------------------------------
 __device__ __forceinline__ float decay_pow(float s2, float n) {
@@ -137,6 +137,33 @@ __device__ __forceinline__ float decay_pow_d(double s2, double n) {
   // Same in double, rounded once; used where a handful of factors per block are tabulated.
   return (float)exp2(-s2 * n);
 }
+
+// four consecutive elements as one vector access, widened to fp32
+template <typename T> struct Vec4;
+template <> struct Vec4<float> {
+  static __device__ __forceinline__ void load(const float* p, float (&x)[4]) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  }
+  static __device__ __forceinline__ void store(float* p, const float (&x)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+  }
+};
+template <> struct Vec4<__nv_bfloat16> {
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&x)[4]) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+    x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+  }
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&x)[4]) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]), b = __floats2bfloat162_rn(x[2], x[3]);
+    uint2 v;
+    v.x = *reinterpret_cast<const uint32_t*>(&a);
+    v.y = *reinterpret_cast<const uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = v;
+  }
+};
 
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
