@@ -225,6 +225,36 @@ la_status la_lrpe_bwd(const la_shape* shape, const void* q, const void* k, const
                       size_t workspace_bytes, void* stream);
 
 /*
+ * One sequence cut into consecutive chunks of chunk_tokens tokens (the last may be shorter), e.g. one chunk per GPU
+ * of a sequence-parallel group.  Only Algorithm 2's d x e state crosses a cut, so the exchange between the chunks'
+ * owners is one gather of [B,H,d,e] fp32 states per direction:
+ *
+ *   la_chunk_state   the chunk's own contribution, from its tokens alone:
+ *                      reverse = 0:  b = k, c = v:    state_out = sum_s lambda^(n-1-s) k_s v_s^T
+ *                                    (what la_fwd would return as kv_out from a zero kv_in);
+ *                      reverse = 1:  b = q, c = d_o:  state_out = sum_t lambda^(t+1) q_t do_t^T
+ *                                    (what la_bwd would return as grad_kv_in for a zero grad_kv_out).
+ *                    shape describes the chunk (N = its tokens).  workspace: la_chunk_state_workspace_bytes(shape),
+ *                    256-byte aligned.
+ *   la_chain_states  the state at a cut from the gathered contributions `states` [num_chunks,B,H,d,e]:
+ *                      reverse = 0:  state_out = the state entering chunk `chunk` (kv_in of its la_fwd / la_bwd),
+ *                                    z = boundary; for j = 0 .. chunk-1: z = lambda^(n_j) z + states[j];
+ *                                    chunk = num_chunks gives the kv_out of the whole sequence;
+ *                      reverse = 1:  state_out = grad_kv_out of chunk `chunk`'s la_bwd,
+ *                                    z = boundary; for j = num_chunks-1 down to chunk+1: z = lambda^(n_j) z + states[j];
+ *                                    chunk = -1 gives the grad_kv_in of the whole sequence.
+ *                    boundary: the whole sequence's kv_in (reverse = 0) or grad_kv_out (reverse = 1), or NULL.
+ *                    shape gives B, H, d, e (N is ignored); total_tokens and chunk_tokens give every n_j.
+ * The results of la_fwd / la_bwd on the chunks with these states are those of the whole sequence on one device.
+ */
+size_t la_chunk_state_workspace_bytes(const la_shape* shape);
+la_status la_chunk_state(const la_shape* shape, int reverse, const void* b, const void* c, const float* lambda_host,
+                         float* state_out, void* workspace, size_t workspace_bytes, void* stream);
+la_status la_chain_states(const la_shape* shape, long long total_tokens, long long chunk_tokens, int reverse,
+                          const float* states, int num_chunks, int chunk, const float* boundary,
+                          const float* lambda_host, float* state_out, void* stream);
+
+/*
  * Packed batches of sequences of different lengths (the serving-side form of Algorithm 2: every sequence has its
  * own state).  The token tensors are [T, H, d] with the num_seqs sequences one after the other: shape->B = 1,
  * shape->N = T, shape->layout = LA_LAYOUT_BNHD; cu_seqlens_host (HOST memory, num_seqs + 1 ints, cu[0] = 0,

@@ -27,7 +27,7 @@ EXPORTS = ("la_workspace_bytes", "la_segment_length", "la_fwd", "la_bwd", "la_de
            "la_status_string", "la_version", "la_launch_count", "la_profile_enable",
            "la_profile_collect", "la_host_arena_bytes", "la_fwd_bwd_host", "la_device_status", "la_fwd_noalloc", "la_bwd_reuse",
            "la_selftest_bounded_wait", "la_fwd_gated", "la_gate_bwd", "la_gate_fwd", "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
-           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd")
+           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd", "la_chunk_state_workspace_bytes", "la_chunk_state", "la_chain_states")
 LA_NOALLOC_SCRATCH_BYTES = 32 << 20
 KERNEL_KINDS = ("prepass", "scan", "walk", "decode", "walk_pair", "gate", "lrpe")
 
@@ -93,6 +93,12 @@ def load():
         lib.la_lrpe_fwd.restype = I
         lib.la_lrpe_bwd.argtypes = [sp, vp, vp, vp, vp, vp, fp, LL, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.la_lrpe_bwd.restype = I
+        lib.la_chunk_state_workspace_bytes.argtypes = [sp]
+        lib.la_chunk_state_workspace_bytes.restype = sz
+        lib.la_chunk_state.argtypes = [sp, I, vp, vp, fp, vp, vp, sz, vp]
+        lib.la_chunk_state.restype = I
+        lib.la_chain_states.argtypes = [sp, LL, LL, I, vp, I, I, vp, fp, vp, vp]
+        lib.la_chain_states.restype = I
         lib.la_decode_steps.argtypes = [sp, vp, vp, vp, fp, vp, vp, vp]
         lib.la_decode_steps.restype = I
         lib.la_host_arena_bytes.argtypes = [sp]
@@ -273,7 +279,7 @@ def la_decode_steps(shape: LaShape, q, k, v, lam, kv, o, stream=None):
                                 _ptr(o), _stream(stream))
     if rc != 0:
         raise LaError(rc, "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
-           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd")
+           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd", "la_chunk_state_workspace_bytes", "la_chunk_state", "la_chain_states")
 
 
 def _cu(cu_seqlens):
@@ -307,7 +313,32 @@ def la_bwd_varlen(shape: LaShape, q, k, v, do, lam, dq, dk, dv, cu_seqlens, kv_i
                               _ptr(dv), cu, S, _ptr(kv_in), _ptr(grad_kv_out), _ptr(grad_kv_in), _ptr(workspace),
                               ws_bytes, _stream(stream))
     if rc != 0:
-        raise LaError(rc, "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd")
+        raise LaError(rc, "la_bwd_varlen")
+
+
+def chunk_state_workspace_bytes(shape: LaShape) -> int:
+    n = load().la_chunk_state_workspace_bytes(ctypes.byref(shape))
+    if n == ctypes.c_size_t(-1).value:
+        raise LaError(2, "la_chunk_state_workspace_bytes")
+    return int(n)
+
+
+def la_chunk_state(shape: LaShape, reverse: int, b, c, lam, state_out, workspace, stream=None):
+    """A chunk's own state contribution: reverse=0 (b=k, c=v) or reverse=1 (b=q, c=dO)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = load().la_chunk_state(ctypes.byref(shape), int(reverse), _ptr(b), _ptr(c), _lam(lam), _ptr(state_out),
+                               _ptr(workspace), ws_bytes, _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_chunk_state")
+
+
+def la_chain_states(shape: LaShape, total_tokens: int, chunk_tokens: int, reverse: int, states, num_chunks: int,
+                    chunk: int, boundary, lam, state_out, stream=None):
+    """The state at a cut from the gathered per-chunk contributions [num_chunks,B,H,d,e]."""
+    rc = load().la_chain_states(ctypes.byref(shape), int(total_tokens), int(chunk_tokens), int(reverse), _ptr(states),
+                                int(num_chunks), int(chunk), _ptr(boundary), _lam(lam), _ptr(state_out), _stream(stream))
+    if rc != 0:
+        raise LaError(rc, "la_chain_states")
 
 
 def lrpe_workspace_bytes(op: int, shape: LaShape) -> int:
@@ -333,7 +364,7 @@ def la_lrpe_bwd(shape: LaShape, q, k, v, do, theta, lam, dq, dk, dv, dtheta, pos
                             _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dtheta), _ptr(kv_in), _ptr(grad_kv_out),
                             _ptr(grad_kv_in), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
-        raise LaError(rc, "la_lrpe_bwd")
+        raise LaError(rc, "la_lrpe_bwd", "la_chunk_state_workspace_bytes", "la_chunk_state", "la_chain_states")
 
 
 def host_arena_bytes(shape: LaShape) -> int:

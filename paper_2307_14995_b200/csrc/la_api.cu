@@ -615,6 +615,82 @@ la_status la_fwd_bwd_host(const la_shape* shape, const void* q_host, const void*
   return LA_OK;
 }
 
+// ---- one sequence cut into chunks (sequence parallelism): the state is all that crosses a cut ---------------------
+size_t la_chunk_state_workspace_bytes(const la_shape* shape) {
+  if (check_shape(shape, true) != LA_OK) return (size_t)-1;
+  Plan p;
+  if (make_plan(shape, &p) != LA_OK) return (size_t)-1;
+  return state_set_bytes(shape, p);
+}
+
+la_status la_chunk_state(const la_shape* shape, int reverse, const void* b, const void* c, const float* lambda_host,
+                         float* state_out, void* workspace, size_t workspace_bytes, void* stream) {
+  la_status st = check_shape(shape, true);
+  if (st != LA_OK) return st;
+  if (!b || !c || !state_out || (reverse != 0 && reverse != 1)) return LA_ERR_INVALID_ARG;
+  if (!aligned16(b) || !aligned16(c) || !aligned16(state_out)) return LA_ERR_INVALID_ARG;
+  DecayTable tab;
+  if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
+  Plan p;
+  if ((st = make_plan(shape, &p)) != LA_OK) return st;
+  const size_t need = state_set_bytes(shape, p);
+  if (!workspace || workspace_bytes < need) return LA_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return LA_ERR_INVALID_ARG;
+  if ((st = check_device()) != LA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  float* buf = static_cast<float*>(workspace);
+  LA_TRY_CUDA(run_prepass(shape, p, tab, b, c, reverse, buf, cs));
+  ChainArgs ca{};
+  ca.src = buf;
+  ca.DE = shape->d * shape->e;
+  ca.stride_j = ca.DE;
+  ca.stride_bh = (long long)p.nseg * ca.DE;
+  ca.z_in = nullptr;
+  ca.out = state_out;
+  ca.BH = p.BH;
+  ca.H = shape->H;
+  ca.first = reverse ? p.nseg - 1 : 0;
+  ca.count = p.nseg;
+  ca.step = reverse ? -1 : 1;
+  ca.N = shape->N;
+  ca.piece_len = p.seg_len;
+  LA_TRY_CUDA(launch_chain(ca, tab, cs));
+  return LA_OK;
+}
+
+la_status la_chain_states(const la_shape* shape, long long total_tokens, long long chunk_tokens, int reverse,
+                          const float* states, int num_chunks, int chunk, const float* boundary,
+                          const float* lambda_host, float* state_out, void* stream) {
+  la_status st = check_shape(shape, false);
+  if (st != LA_OK) return st;
+  if (!states || !state_out || (reverse != 0 && reverse != 1)) return LA_ERR_INVALID_ARG;
+  if (!aligned16(states) || !aligned16(state_out) || !aligned16(boundary)) return LA_ERR_INVALID_ARG;
+  if (num_chunks < 1 || chunk_tokens < 1 || total_tokens < 1) return LA_ERR_INVALID_ARG;
+  if ((total_tokens + chunk_tokens - 1) / chunk_tokens != num_chunks) return LA_ERR_INVALID_ARG;
+  // forward: the state entering chunk `chunk` (0 .. num_chunks; num_chunks = after the last chunk);
+  // reverse: the state gradient entering chunk `chunk` from the right (-1 .. num_chunks - 1; -1 = before the first)
+  if (reverse ? (chunk < -1 || chunk > num_chunks - 1) : (chunk < 0 || chunk > num_chunks)) return LA_ERR_INVALID_ARG;
+  DecayTable tab;
+  if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
+  if ((st = check_device()) != LA_OK) return st;
+  ChainArgs ca{};
+  ca.src = states;
+  ca.DE = shape->d * shape->e;
+  ca.BH = shape->B * shape->H;
+  ca.stride_j = (long long)ca.BH * ca.DE;
+  ca.stride_bh = ca.DE;
+  ca.z_in = boundary;
+  ca.out = state_out;
+  ca.H = shape->H;
+  ca.first = reverse ? num_chunks - 1 : 0;
+  ca.count = reverse ? num_chunks - 1 - chunk : chunk;
+  ca.step = reverse ? -1 : 1;
+  ca.N = total_tokens;
+  ca.piece_len = chunk_tokens;
+  LA_TRY_CUDA(launch_chain(ca, tab, static_cast<cudaStream_t>(stream)));
+  return LA_OK;
+}
+
 // ---- packed batches of sequences of different lengths -------------------------------------------------------
 namespace {
 // Checks the packed description and returns, through `sub`, the shape of one sequence (N filled in per sequence).

@@ -67,6 +67,20 @@ struct ScanArgs {
   int BH, H, N, seg_len, nseg, Da, Ec, reverse;
 };
 
+// Chain of piece-local states into the state at one boundary (a cut of the sequence):
+//   forward (first <= last):  z = z_in;  for j = first .. last:      z = lambda^(L_j) z + src_j
+//   reverse (first >  last):  z = z_in;  for j = first down to last: z = lambda^(L_j) z + src_j
+// with L_j = tokens of piece j = min(N, (j+1) piece_len) - j piece_len.  count == 0 copies z_in (or zeros).
+struct ChainArgs {
+  const float* src;         // element i of piece j of (b,h): src[j * stride_j + bh * stride_bh + i]
+  long long stride_j, stride_bh;
+  const float* z_in;        // [BH, DE] or NULL = zeros
+  float* out;               // [BH, DE]
+  int BH, H, DE;
+  int first, count, step;   // pieces first, first + step, ... (count of them), step = +1 or -1
+  long long N, piece_len;
+};
+
 // dtype tags as in la.h
 enum { DT_BF16 = 0, DT_F32 = 1 };
 
@@ -76,6 +90,7 @@ cudaError_t launch_simt_walk(const OpArgs& args, const DecayTable& tab, int Da, 
 cudaError_t launch_simt_prepass(const OpArgs& args, const DecayTable& tab, int Da, int Ec, int in_dt,
                                 cudaStream_t stream);
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream);
+cudaError_t launch_chain(const ChainArgs& args, const DecayTable& tab, cudaStream_t stream);
 // dst[m] = transpose(src[m]) for `count` row-major Da x Ec fp32 matrices.
 cudaError_t launch_transpose_states(const float* src, float* dst, long count, int Da, int Ec, cudaStream_t stream);
 // T >= 1 consecutive tokens per (batch, head); token t of (b,h) is the row at element offset b*sB + h*sH + t*sT.

@@ -452,6 +452,40 @@ cudaError_t launch_transpose_states(const float* src, float* dst, long count, in
   return cudaGetLastError();
 }
 
+// One thread per four consecutive state elements; the pieces are few (ranks of a sequence-parallel group, or the
+// segments of one chunk), so the sequential chain is short and every access is a coalesced 16-byte one.
+__global__ void __launch_bounds__(256) chain_kernel(const ChainArgs args, const DecayTable tab) {
+  const long per_head = args.DE / 4;
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long)args.BH * per_head) return;
+  const int bh = (int)(i / per_head);
+  const size_t e0 = (size_t)(i % per_head) * 4;
+  const double s2 = tab.s2[bh % args.H];
+  float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (args.z_in) z = *reinterpret_cast<const float4*>(args.z_in + (size_t)bh * args.DE + e0);
+  int j = args.first;
+  for (int n = 0; n < args.count; ++n, j += args.step) {
+    const long long t0 = (long long)j * args.piece_len;
+    const long long t1 = (t0 + args.piece_len < args.N) ? t0 + args.piece_len : args.N;
+    const float g = decay_pow_d(s2, (double)(t1 - t0));
+    const float4 x = *reinterpret_cast<const float4*>(args.src + (size_t)j * args.stride_j + (size_t)bh * args.stride_bh + e0);
+    z.x = fmaf(g, z.x, x.x);
+    z.y = fmaf(g, z.y, x.y);
+    z.z = fmaf(g, z.z, x.z);
+    z.w = fmaf(g, z.w, x.w);
+  }
+  *reinterpret_cast<float4*>(args.out + (size_t)bh * args.DE + e0) = z;
+}
+
+cudaError_t launch_chain(const ChainArgs& args, const DecayTable& tab, cudaStream_t stream) {
+  if (args.DE % 4 != 0 || args.BH < 1 || args.count < 0 || args.piece_len < 1) return cudaErrorInvalidValue;
+  const long threads = (long)args.BH * (args.DE / 4);
+  KernelTimer timer(K_SCAN, stream);
+  chain_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(args, tab);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_scan(const ScanArgs& args, const DecayTable& tab, cudaStream_t stream) {
   if (args.nseg > SCAN_MAX_SEG || (args.Da % 32) != 0 || (args.Ec % 32) != 0) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)args.BH, (unsigned)((args.Da / 32) * (args.Ec / 32)));
