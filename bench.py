@@ -390,6 +390,23 @@ def run_ours(args):
                 "workspace_bytes": {"fwd": wl_f.numel(), "bwd": wl_b.numel()}}
         del wl_f, wl_b, theta, dth
 
+    # ---- sequence parallelism: what one rank adds around its la_fwd / la_bwd when the shape is one chunk of a longer
+    # sequence (the all-gather itself needs more than one GPU and is not timed here) ----
+    seqpar_leg = None
+    if train_steps and args.only == "all":
+        st_loc = torch.empty((w.B, w.H, w.d, w.e), dtype=torch.float32, device=dev)
+        st_all = torch.zeros((8, w.B, w.H, w.d, w.e), dtype=torch.float32, device=dev)
+        ws_s = torch.empty(max(la.chunk_state_workspace_bytes(shape), 256), dtype=torch.uint8, device=dev)
+        cs_f, _ = time_loop(lambda: la.la_chunk_state(shape, 0, k, v, lam, st_loc, ws_s, stream))
+        cs_r, _ = time_loop(lambda: la.la_chunk_state(shape, 1, q, do, lam, st_loc, ws_s, stream))
+        ch, _ = time_loop(lambda: la.la_chain_states(shape, 8 * w.N, w.N, 0, st_all, 8, 7, None, lam, st_loc, stream))
+        seqpar_leg = {"what": "per-rank additions of the sequence-parallel protocol at this shape as one chunk of 8: "
+                              "la_chunk_state (forward: k, v; reverse: q, dO), la_chain_states over 7 earlier chunks",
+                      "chunk_state_fwd_ms": cs_f, "chunk_state_rev_ms": cs_r, "chain_ms": ch,
+                      "gathered_bytes_per_rank_and_direction": st_loc.numel() * 4,
+                      "added_fraction_of_step": (cs_f + cs_r + 2 * ch) / ms_step}
+        del st_loc, st_all, ws_s
+
     # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
     dw = inputs.WORKLOADS["decode"]
     gen = torch.Generator(dev)
@@ -548,7 +565,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / prof_steps for kname, (ms, _) in prof.items()},
             "kernel_launches_per_step": {kname: c / prof_steps for kname, (_, c) in prof.items()},
-            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe,
+            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe, "sequence_parallel": seqpar_leg,
             "roofline": {"scope": "ONE kernel, the dominant one; the whole-step figure the target is stated on is step_roofline",
                          "kernel": "full-width block walk (tc_walk_full_kernel), single-job launches (O and dQ)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -1,6 +1,10 @@
 // Tensor-core kernels of the generic decayed linear-attention operator for
-// bf16 inputs with Da = Ec = D, D = 128 or 64 (block formulas: la_common.cuh; the text below is for
-// D = 128, the differences at D = 64 are described at the kernel's template parameter).
+// bf16 inputs with Da = Ec = D, D = 128 or 64 (block formulas: la_common.cuh).  Two kernels share this file's
+// launchers: the half-width kernel below (every D = 64 launch, the state-only pre-pass at both head sizes, and the
+// D = 128 walk when an output is aligned to 16 but not 32 bytes) and the full-width walk of la_tc_full.cuh
+// (D = 128: one thread block per (batch*head, segment) with all four 128x128 accumulators in tensor memory),
+// which launch_walk_d prefers.  The text below describes the half-width kernel at D = 128; the differences at
+// D = 64 are described at the kernel's template parameter.
 //
 // One thread block walks the 128-token blocks of one (batch*head, segment,
 // half of the value columns).  Per block it issues, on the 5th-generation
@@ -24,7 +28,9 @@
 // Warp roles (24 warps; every group has whole multiples of four warps because a warp
 // can only touch the 32-lane quarter of tensor memory given by its index mod 4):
 //   warp 0       TMA producer: a, b, c tiles into a 2-stage shared-memory ring
-//   warp 1       owns tensor memory, issues every MMA from one lane
+//   warp 1       owns tensor memory and issues every MMA: the whole warp stays converged through the waits and
+//                one elected lane issues each group of eight K-steps (a lone lane looping over the products
+//                was measurably slower: its barrier polls and descriptor arithmetic did not overlap)
 //   warps 4-11   "P" group (two warps per quarter, two 32-column chunks each): S (fp32) ->
 //                masked, decayed P as packed bf16 hi/lo, written back over S in tensor
 //                memory, where M4 reads it as its A operand
@@ -36,14 +42,14 @@
 // In the state-only pre-pass warps 4-19 all form fc, and the MMA warp issues converged.
 // All hand-offs are mbarriers; every wait is bounded and an expired wait makes the whole
 // block unwind (flag set, copies drained, tensor memory freed).  Barrier operations on the MMA
-// lane are kept few, since each costs the lane about a hundred clocks (measured): per block it
+// warp are kept few, since each costs it a few hundred clocks (measured): per block it
 // waits for Z_READY (state operand and fc, both written by the Z group), FULL_B of the next block
 // (a and b tiles travel together), P_READY (P written AND the previous block's accumulators read
 // by the output group: 8 + 4 arrivals) and FULL_C, and commits to DZ_READY, A_FREE (which the
 // producer and the Z group both wait for), S_READY and O_READY.
 //
 // The only chain that is sequential across blocks is dZ -> Z -> O_inter; S, P and fc of
-// block n+1 do not depend on block n.  The MMA lane therefore issues, per block n:
+// block n+1 do not depend on block n.  The MMA warp therefore issues, per block n:
 // M3(n), M2(n), M1(n+1), M4(n): the state chain first (it never waits for a load), then the
 // next score tile so that the P group always has work, then the product that needs P.
 //

@@ -376,7 +376,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
     // the rows for a bulk store).  A thread holds one row, so a plain store instruction would touch 32 different
     // lines, and the load/store unit's time per line is what the other groups' shared-memory traffic then waits
     // behind (measured: 2048 line accesses per block cost 2500 clocks of a 9100-clock block, 512 cost 700).  So each
-    // 128-byte piece of four rows is first transposed among four lanes with two rounds of shuffles: afterwards lane
+    // 128-byte piece of four rows is first transposed among four lanes with two exchanges by shuffles: afterwards lane
     // g of a quad holds the g-th 32 bytes of its quad's four rows, and one store instruction writes whole 128-byte
     // lines (8 rows per instruction instead of 32 quarter-lines).
     const int q = warp & 3;
@@ -451,7 +451,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
             }
           }
         }
-        // round 1, partner lane ^ 1: the even lane keeps chunks 0 and 2 and sends 1 and 3, the odd lane the other way
+        // first exchange, partner lane ^ 1: the even lane keeps chunks 0 and 2 and sends 1 and 3, the odd lane the other way
         // round; afterwards chunk slots hold (own row, chunk b0), (partner row, chunk b0), (own, 2 + b0), (partner, 2 + b0)
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
@@ -462,7 +462,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
           w[16 + x] = k2;
           w[24 + x] = __shfl_xor_sync(0xffffffffu, s2x, 1);
         }
-        // round 2, partner lane ^ 2: lanes 0, 1 of the quad keep the chunk-b0 pair and send the chunk-(2 + b0) pair,
+        // second exchange, partner lane ^ 2: lanes 0, 1 of the quad keep the chunk-b0 pair and send the chunk-(2 + b0) pair,
         // lanes 2, 3 the other way round; afterwards slot k holds chunk g of the row of lane ^ k
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
