@@ -103,7 +103,8 @@ typedef struct {
 
 /* Bytes of device scratch the given op needs for this shape (0 is possible).
  * Returns (size_t)-1 if the shape is invalid or unsupported.  Linear in
- * B*H*d*e*ceil(N/seg_len); never grows with N^2. */
+ * B*H*d*e*ceil(N/seg_len); never grows with N^2: sets of [B,H,nseg,d,e] fp32 states,
+ * two for the forward pass (0 with a single segment), three for the backward pass. */
 size_t la_workspace_bytes(int op, const la_shape* shape);
 
 /* The segment length the library will use for this shape (after applying
@@ -119,7 +120,7 @@ int la_segment_length(const la_shape* shape);
  * workspace: device scratch of at least la_workspace_bytes(LA_OP_FWD, shape)
  * bytes, 256-byte aligned; may be NULL when that size is 0.  Calls that share a
  * workspace must be stream-ordered.  Afterwards the workspace holds the state
- * entering each segment; la_bwd_reuse can take it to skip recomputing those.
+ * entering each segment and its transpose; la_bwd_reuse can take it to skip recomputing those.
  */
 la_status la_fwd(const la_shape* shape, const void* q, const void* k, const void* v,
                  const float* lambda_host, void* o, const float* kv_in, float* kv_out,

@@ -249,7 +249,7 @@ size_t la_workspace_bytes(int op, const la_shape* shape) {
   Plan p;
   if (make_plan(shape, &p) != LA_OK) return (size_t)-1;
   const size_t one = state_set_bytes(shape, p);
-  if (op == LA_OP_FWD) return p.nseg > 1 ? one : 0;
+  if (op == LA_OP_FWD) return p.nseg > 1 ? 2 * one : 0;  // the states entering each segment, and their transposes
   return 3 * one;
 }
 
@@ -316,7 +316,8 @@ la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const vo
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
   Plan p;
   if ((st = make_plan(shape, &p)) != LA_OK) return st;
-  const size_t need = p.nseg > 1 ? state_set_bytes(shape, p) : 0;
+  const size_t one = state_set_bytes(shape, p);
+  const size_t need = p.nseg > 1 ? 2 * one : 0;
   if (need > 0 && (!workspace || workspace_bytes < need)) return LA_ERR_WORKSPACE;
   if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return LA_ERR_INVALID_ARG;
   if ((st = check_device()) != LA_OK) return st;
@@ -326,7 +327,8 @@ la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const vo
   if (p.nseg > 1) {
     float* buf = static_cast<float*>(workspace);
     LA_TRY_CUDA(run_prepass(shape, p, tab, k, v, 0, buf, cs));
-    LA_TRY_CUDA(run_scan(shape, p, tab, buf, nullptr, kv_in, false, 0, cs));
+    // the transposed copy (second set) is what the dQ walk of la_bwd_reuse starts from
+    LA_TRY_CUDA(run_scan(shape, p, tab, buf, buf + one / sizeof(float), kv_in, false, 0, cs));
     entry = buf;
   }
   if (!u) {
@@ -391,10 +393,8 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
   // dQ = fwd(a = dO, b = V, c = K); its state is KV^T, so the caller's kv_in enters transposed.
   const float* entry_q = nullptr;
   if (multi && fwd_workspace) {
-    // la_fwd left KV entering each segment (kv_in included) in its workspace: transpose, no pre-pass
-    LA_TRY_CUDA(launch_transpose_states(static_cast<const float*>(fwd_workspace), buf_kvt, (long)p.BH * p.nseg,
-                                        shape->d, shape->e, cs));
-    entry_q = buf_kvt;
+    // la_fwd left KV entering each segment (kv_in included) and its transpose in its workspace: no pre-pass, no scan
+    entry_q = static_cast<const float*>(fwd_workspace) + one / sizeof(float);
   } else if (multi || kv_in) {
     if (multi) LA_TRY_CUDA(run_prepass(shape, p, tab, v, k, 0, buf_kvt, cs));
     LA_TRY_CUDA(run_scan(shape, p, tab, buf_kvt, nullptr, kv_in, true, 0, cs));

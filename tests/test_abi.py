@@ -54,13 +54,13 @@ def test_workspace_is_linear_in_segments_not_quadratic(lib):
     seg = la.segment_length(s1)
     assert seg % 128 == 0 and seg >= 1024
     nseg = -(-65536 // seg)
-    assert la.workspace_bytes(la.LA_OP_FWD, s1) == 32 * nseg * 128 * 128 * 4
+    assert la.workspace_bytes(la.LA_OP_FWD, s1) == 2 * 32 * nseg * 128 * 128 * 4
     assert la.workspace_bytes(la.LA_OP_BWD, s1) == 3 * 32 * nseg * 128 * 128 * 4
     assert la.workspace_bytes(la.LA_OP_DECODE, s1) == 0
     s2 = shape(N=100)
     assert la.workspace_bytes(la.LA_OP_FWD, s2) == 0  # one segment: no scratch at all
     s3 = shape(N=1000, seg_len=128)
-    assert la.workspace_bytes(la.LA_OP_FWD, s3) == 2 * 8 * 64 * 64 * 4
+    assert la.workspace_bytes(la.LA_OP_FWD, s3) == 2 * 2 * 8 * 64 * 64 * 4
 
 
 @pytest.mark.parametrize("bad", [dict(d=48, e=48), dict(d=64, e=128), dict(H=300),

@@ -16,10 +16,10 @@ from paper_2307_14995_b200 import binding as la, inputs
 
 
 def test_noalloc_rejects_shapes_beyond_the_static_scratch():
-    # 64 heads x 8 segments x 64 KB = 32 MiB fits exactly; one more segment does not.
+    # 64 heads x 4 segments x 2 sets x 64 KB = 32 MiB fits exactly; one more segment does not.
     la.load()
-    fits = la.make_shape(1, 64, 8 * 128, 128, 128, torch.bfloat16, torch.float32, seg_len=128, path=la.LA_PATH_SIMT)
-    too_big = la.make_shape(1, 64, 9 * 128, 128, 128, torch.bfloat16, torch.float32, seg_len=128, path=la.LA_PATH_SIMT)
+    fits = la.make_shape(1, 64, 4 * 128, 128, 128, torch.bfloat16, torch.float32, seg_len=128, path=la.LA_PATH_SIMT)
+    too_big = la.make_shape(1, 64, 5 * 128, 128, 128, torch.bfloat16, torch.float32, seg_len=128, path=la.LA_PATH_SIMT)
     assert la.workspace_bytes(la.LA_OP_FWD, fits) == la.LA_NOALLOC_SCRATCH_BYTES
     assert la.workspace_bytes(la.LA_OP_FWD, too_big) > la.LA_NOALLOC_SCRATCH_BYTES
     lam = (ctypes.c_float * 64)(*([0.5] * 64))
