@@ -78,8 +78,8 @@ constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_OI = 256, COL_OE0 = 320, COL_OE
 constexpr long long WAIT_BUDGET = 2000000000LL;  // clocks (~1 s)
 
 enum Bar {
-  FULL_B0 = 0, FULL_B1, FULL_C0, FULL_C1,                     // TMA -> consumers (FULL_B: b, and a in the walk kernel)
-  A_FREE0, A_FREE1, B_FREE0, B_FREE1, C_FREE0, C_FREE1,       // consumers -> TMA
+  FULL_B0 = 0, FULL_B1, FULL_B2, FULL_C0, FULL_C1, FULL_C2,   // TMA -> consumers (FULL_B: b, and a in the walk kernel)
+  A_FREE0, A_FREE1, B_FREE0, B_FREE1, B_FREE2, C_FREE0, C_FREE1, C_FREE2,  // consumers -> TMA (third stage: state-only kernel)
   S_READY0, S_READY1, P_READY0, P_READY1,
   FC_READY0, FC_READY1, FC_FREE0, FC_FREE1,                   // (second buffer: state-only kernel)
   DZ_READY, Z_READY, O_READY, OG_SYNC, DRAIN,
@@ -294,7 +294,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
       if (i == P_READY0 || i == P_READY1) count = 12;
       if (i == OG_SYNC) count = 4;
       // the c tile is released by the warps that read it (state-only) / by the thread that stores from it (walk)
-      if (i == C_FREE0 || i == C_FREE1) count = STATE_ONLY ? 16 : 1;
+      if (i == C_FREE0 || i == C_FREE1 || i == C_FREE2) count = STATE_ONLY ? 16 : 1;
       mbar_init(&sm.bars[i], count);
     }
     sm.abort = 0;
@@ -311,6 +311,9 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
   if (D == 64) {
     for (int i = tid; i < 2 * 1024; i += TC_THREADS)
       reinterpret_cast<uint4*>(&sm.st[i >> 10].b[1][0])[i & 1023] = make_uint4(0u, 0u, 0u, 0u);
+    if (STATE_ONLY)  // the third load stage keeps its b tile where the walk kernel has stage 0's a tile
+      for (int i = tid; i < 1024; i += TC_THREADS)
+        reinterpret_cast<uint4*>(&sm.st[0].a[1][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
   }
   tc_fence_before_sync();
@@ -319,32 +322,38 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
   const uint32_t tmem = sm.tmem_slot;
   bool issued_mma = false;
   uint32_t mma_elected = 0;  // set in the lane of warp 1 that issues the tensor-core instructions
-  int armed_b[2] = {0, 0}, armed_c[2] = {0, 0};  // producer: uses armed per stage
+  int armed_b[3] = {0, 0, 0}, armed_c[3] = {0, 0, 0};  // producer: uses armed per stage
+  // State-only kernel: three load stages (the a tiles, which it never loads, hold the third stage's b and c), so
+  // that a thread block running alone at the end of the launch has 144 KB in flight instead of 96 KB: its time per
+  // block is the latency of HBM divided by the stages in flight.  The fc buffers stay two deep (it & 1).
+  constexpr int NLS = STATE_ONLY ? 3 : 2;
+  auto b_tile = [&](int ls) { return ls == 0 ? &sm.st[0].b[0][0] : (ls == 1 ? &sm.st[1].b[0][0] : &sm.st[0].a[0][0]); };
+  auto c_tile = [&](int ls) { return ls == 0 ? &sm.st[0].c[0] : (ls == 1 ? &sm.st[1].c[0] : &sm.st[1].a[0][0]); };
 
   if (warp == 0) {
     // ------------------------------------ TMA producer ------------------------------------
     if (lane == 0) {
       for (int it = 0; it < nblk; ++it) {
-        const int s = it & 1;
-        const uint32_t prev = ((it >> 1) - 1) & 1;  // parity of this stage's previous use
+        const int s = STATE_ONLY ? it % NLS : (it & 1);
+        const int use = STATE_ONLY ? it / NLS : (it >> 1);  // how often this stage has been used before
+        const uint32_t prev = (use - 1) & 1;                // parity of this stage's previous use
         const int blk = REV ? (nblk - 1 - it) : (it + it0);
         const int t0 = seg_t0 + blk * 128;
-        Stage& stg = sm.st[s];
-        // State-only kernel: its two stages hold less than what must be in flight to cover the latency of
-        // HBM, so the tiles two blocks ahead are pulled into L2 now and the loads proper become L2 hits
-        // (measured: 0.276 -> 0.245 ms per launch; the same in the walk kernel made it slower).
-        if (STATE_ONLY && it + 2 < nblk) {
-          const int tp = seg_t0 + (REV ? (nblk - 3 - it) : (it + 2 + it0)) * 128;
+        // State-only kernel: the tiles a few blocks ahead are pulled into L2 now, so that the loads proper are
+        // L2 hits (measured: 0.276 -> 0.245 ms per launch; the same in the walk kernel made it slower).
+        if (STATE_ONLY && it + NLS < nblk) {
+          const int tp = seg_t0 + (REV ? (nblk - 1 - NLS - it) : (it + NLS + it0)) * 128;
           tma_prefetch_4d(tm_b, 0, tp, hh_, bb_);
           if (D == 128) tma_prefetch_4d(tm_b, 64, tp, hh_, bb_);
           tma_prefetch_4d(tm_c, ehalf * 64, tp, hh_, bb_);
         }
         if (STATE_ONLY) {
-          if (it >= 2) TC_WAIT(B_FREE0 + s, prev, 1);
+          if (it >= NLS) TC_WAIT(B_FREE0 + s, prev, 1);
           mbar_arrive_expect_tx(&sm.bars[FULL_B0 + s], D * 256);
-          tma_load_4d(&stg.b[0][0], tm_b, &sm.bars[FULL_B0 + s], 0, t0, hh_, bb_);
-          if (D == 128) tma_load_4d(&stg.b[1][0], tm_b, &sm.bars[FULL_B0 + s], 64, t0, hh_, bb_);
+          tma_load_4d(b_tile(s), tm_b, &sm.bars[FULL_B0 + s], 0, t0, hh_, bb_);
+          if (D == 128) tma_load_4d(b_tile(s) + 128 * 64, tm_b, &sm.bars[FULL_B0 + s], 64, t0, hh_, bb_);
         } else {
+          Stage& stg = sm.st[s];
           // walk kernel: the a and b tiles of a stage travel together (one barrier for both, FULL_B); A_FREE
           // is committed after M2, the last product of the block that reads either of them
           if (it >= 2) TC_WAIT(A_FREE0 + s, prev, 3);
@@ -354,11 +363,11 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
           tma_load_4d(&stg.a[0][0], tm_a, &sm.bars[FULL_B0 + s], 0, t0, hh_, bb_);
           if (D == 128) tma_load_4d(&stg.a[1][0], tm_a, &sm.bars[FULL_B0 + s], 64, t0, hh_, bb_);
         }
-        armed_b[s] = (it >> 1) + 1;
-        if (it >= 2) TC_WAIT(C_FREE0 + s, prev, 2);
+        armed_b[s] = use + 1;
+        if (it >= NLS) TC_WAIT(C_FREE0 + s, prev, 2);
         mbar_arrive_expect_tx(&sm.bars[FULL_C0 + s], 16384);
-        tma_load_4d(&stg.c[0], tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, hh_, bb_);
-        armed_c[s] = (it >> 1) + 1;
+        tma_load_4d(c_tile(s), tm_c, &sm.bars[FULL_C0 + s], ehalf * 64, t0, hh_, bb_);
+        armed_c[s] = use + 1;
       }
     }
   } else if (warp == 1 && STATE_ONLY) {
@@ -374,14 +383,16 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
       const uint32_t go = elect_one();
       mma_elected = go;
       // low descriptor halves (MN-major: 64-element chunks 16 KB apart); K step k adds k * 2 KB >> 4
-      const uint32_t bm0 = umma_desc_lo(smem_u32(&sm.st[0].b[0][0]), 16384), bm1 = umma_desc_lo(smem_u32(&sm.st[1].b[0][0]), 16384);
+      const uint32_t bm0 = umma_desc_lo(smem_u32(b_tile(0)), 16384), bm1 = umma_desc_lo(smem_u32(b_tile(1)), 16384);
+      const uint32_t bm2 = umma_desc_lo(smem_u32(b_tile(2)), 16384);
       const uint32_t fh_lo = umma_desc_lo(smem_u32(&sm.fc_hi[0]), 16384), zh_lo = umma_desc_lo(smem_u32(&sm.z_hi[0]), 16384);
       for (int it = 0; it < nblk; ++it) {
-        const int s = it & 1;
+        const int ls = it % NLS;   // load stage of the b tile
+        const int s = it & 1;      // fc buffer
         const uint32_t par2 = (it >> 1) & 1;
-        const uint32_t bm = s ? bm1 : bm0;
+        const uint32_t bm = ls == 0 ? bm0 : (ls == 1 ? bm1 : bm2);
         const uint32_t fbuf_lo = s ? zh_lo : fh_lo;  // fc buffer of this iteration (hi then lo, 16 KB apart)
-        TC_WAIT_WARP(FULL_B0 + s, par2, 4);
+        TC_WAIT_WARP(FULL_B0 + ls, (it / NLS) & 1, 4);
         TC_WAIT_WARP(FC_READY0 + s, par2, 5);
         tc_fence_after_sync();
         // tensor memory is otherwise unused here, so hi and lo share one N = 128 instruction
@@ -391,7 +402,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
           umma_bf16_lh(tmem + COL_S0, bm + k * 128, fbuf_lo + k * 128, HI, split_c ? ID_MN128 : ID_MN64,
                        (it > 0 || k > 0), go);
         issued_mma = true;
-        umma_commit_if(&sm.bars[B_FREE0 + s], go);
+        umma_commit_if(&sm.bars[B_FREE0 + ls], go);
         umma_commit_if(&sm.bars[FC_FREE0 + s], go);
       }
       umma_commit_if(&sm.bars[DZ_READY], go);
@@ -465,9 +476,10 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
       float f = 0.f;
       if (r < min(128, seg_t1 - t0))
         f = REV ? exp2f(-s2 * (float)(t0 + r - seg_t0 + 1)) : exp2f(-s2 * (float)(seg_t1 - 1 - t0 - r));
-      TC_WAIT_WARP(FULL_C0 + s, (it >> 1) & 1, 18);
+      const int ls = it % NLS;  // load stage of the c tile
+      TC_WAIT_WARP(FULL_C0 + ls, (it / NLS) & 1, 18);
       if (it >= 2) TC_WAIT_WARP(FC_FREE0 + s, ((it >> 1) - 1) & 1, 19);  // the MMA two blocks back has read this buffer
-      const __nv_bfloat16* ctile = &sm.st[s].c[0];
+      const __nv_bfloat16* ctile = c_tile(ls);
       __nv_bfloat16* hi_tile = s ? sm.z_hi : sm.fc_hi;
       __nv_bfloat16* lo_tile = s ? sm.z_lo : sm.fc_lo;
 #pragma unroll
@@ -489,7 +501,7 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
       }
       fence_proxy_async_smem();
       WARP_ARRIVE(FC_READY0 + s);
-      if (lane == 0) mbar_arrive(&sm.bars[C_FREE0 + s]);
+      if (lane == 0) mbar_arrive(&sm.bars[C_FREE0 + ls]);
     }
     if (warp >= 12) {
       // segment-local state = accumulated dZ (hi-part + lo-part); this warp's 32 state columns of row r
@@ -784,7 +796,7 @@ teardown:
   // block exits (loads into shared memory, tensor-core work on tensor memory).
   if (sm.abort) {
     if (warp == 0 && lane == 0) {
-      for (int s = 0; s < 2; ++s) {
+      for (int s = 0; s < 3; ++s) {
         if (armed_b[s] > 0) drain_wait(&sm.bars[FULL_B0 + s], (armed_b[s] - 1) & 1);
         if (armed_c[s] > 0) drain_wait(&sm.bars[FULL_C0 + s], (armed_c[s] - 1) & 1);
       }
