@@ -278,8 +278,7 @@ def la_decode_steps(shape: LaShape, q, k, v, lam, kv, o, stream=None):
     rc = load().la_decode_steps(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _lam(lam), _ptr(kv),
                                 _ptr(o), _stream(stream))
     if rc != 0:
-        raise LaError(rc, "la_decode_steps", "la_varlen_workspace_bytes", "la_fwd_varlen",
-           "la_bwd_varlen", "la_lrpe_workspace_bytes", "la_lrpe_fwd", "la_lrpe_bwd", "la_chunk_state_workspace_bytes", "la_chunk_state", "la_chain_states")
+        raise LaError(rc, "la_decode_steps")
 
 
 def _cu(cu_seqlens):
@@ -364,7 +363,7 @@ def la_lrpe_bwd(shape: LaShape, q, k, v, do, theta, lam, dq, dk, dv, dtheta, pos
                             _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dtheta), _ptr(kv_in), _ptr(grad_kv_out),
                             _ptr(grad_kv_in), _ptr(workspace), ws_bytes, _stream(stream))
     if rc != 0:
-        raise LaError(rc, "la_lrpe_bwd", "la_chunk_state_workspace_bytes", "la_chunk_state", "la_chain_states")
+        raise LaError(rc, "la_lrpe_bwd")
 
 
 def host_arena_bytes(shape: LaShape) -> int:
