@@ -407,6 +407,43 @@ def run_ours(args):
                       "added_fraction_of_step": (cs_f + cs_r + 2 * ch) / ms_step}
         del st_loc, st_all, ws_s
 
+    # ---- packed batch of sequences of different lengths (prefill of a serving batch), forward only ----
+    varlen_leg = None
+    if train_steps and args.only == "all":
+        gen_v = torch.Generator("cpu")
+        gen_v.manual_seed(5)
+        lens = [int(x) for x in torch.randint(64, 4097, (64,), generator=gen_v)]
+        cu = [0]
+        for n_ in lens:
+            cu.append(cu[-1] + n_)
+        Tt = cu[-1]
+        vshape = la.make_shape(1, w.H, Tt, w.d, w.e, torch.bfloat16, out_dtype, layout=la.LA_LAYOUT_BNHD)
+        gen_d = torch.Generator(dev)
+        gen_d.manual_seed(6 + rank)
+        vq = torch.nn.functional.silu(torch.randn((1, Tt, w.H, w.d), generator=gen_d, device=dev)).to(torch.bfloat16)
+        vk = torch.nn.functional.silu(torch.randn((1, Tt, w.H, w.d), generator=gen_d, device=dev)).to(torch.bfloat16)
+        vv = torch.randn((1, Tt, w.H, w.e), generator=gen_d, device=dev).to(torch.bfloat16)
+        vo = torch.empty((1, Tt, w.H, w.e), dtype=out_dtype, device=dev)
+        vkv = torch.empty((len(lens), w.H, w.d, w.e), dtype=torch.float32, device=dev)
+        vws = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_FWD, vshape, cu), 256), dtype=torch.uint8, device=dev)
+        pk_ms, pk_l = time_loop(lambda: la.la_fwd_varlen(vshape, vq, vk, vv, lam, vo, cu, None, vkv, vws, stream))
+
+        def one_by_one():
+            for i_ in range(len(lens)):
+                a_, b_ = cu[i_], cu[i_ + 1]
+                sh_ = la.make_shape(1, w.H, b_ - a_, w.d, w.e, torch.bfloat16, out_dtype, layout=la.LA_LAYOUT_BNHD)
+                la.la_fwd(sh_, vq[:, a_:b_], vk[:, a_:b_], vv[:, a_:b_], lam, vo[:, a_:b_], None, vkv[i_:i_ + 1], vws, stream)
+
+        sq_ms, sq_l = time_loop(one_by_one, n=3)
+        eb = 4 if out_dtype == torch.float32 else 2
+        vbytes = Tt * w.H * (3 * 2 * w.d + eb * w.e)
+        varlen_leg = {"what": "la_fwd_varlen over 64 packed sequences of 64..4096 tokens (seeded lengths), %d tokens, H=%d, "
+                              "d=e=%d: all sequences in one set of launches, against one la_fwd per sequence" % (Tt, w.H, w.d),
+                      "packed_ms": pk_ms, "packed_launches": pk_l, "packed_gbs": vbytes / (pk_ms * 1e-3) / 1e9,
+                      "frac_of_hbm_peak": vbytes / (pk_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                      "per_sequence_ms": sq_ms, "per_sequence_launches": sq_l, "tokens": Tt}
+        del vq, vk, vv, vo, vkv, vws
+
     # ---- decode leg: prefill once, then timed recurrent steps on the fp32 state ----
     dw = inputs.WORKLOADS["decode"]
     gen = torch.Generator(dev)
@@ -565,7 +602,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / prof_steps for kname, (ms, _) in prof.items()},
             "kernel_launches_per_step": {kname: c / prof_steps for kname, (_, c) in prof.items()},
-            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe, "sequence_parallel": seqpar_leg,
+            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe, "sequence_parallel": seqpar_leg, "varlen_prefill": varlen_leg,
             "roofline": {"scope": "ONE kernel, the dominant one; the whole-step figure the target is stated on is step_roofline",
                          "kernel": "full-width block walk (tc_walk_full_kernel), single-job launches (O and dQ)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -262,8 +262,11 @@ la_status la_chain_states(const la_shape* shape, long long total_tokens, long lo
  * cu[num_seqs] = T, strictly increasing) gives the first token of each sequence.  Sequence i runs
  * from the state kv_in[i] (or zero) and leaves kv_out[i]; kv_in, kv_out, grad_kv_out, grad_kv_in are
  * [num_seqs, H, d, e] fp32 or NULL.  Results are those of la_fwd / la_bwd on each sequence alone.
- * This version enqueues one la_fwd / la_bwd per sequence on `stream` (3 and 8 launches each), which suits a
- * few long sequences; the workspace is shared: la_varlen_workspace_bytes gives the largest need of any sequence.
+ * bf16 inputs at d = e = 128 with outputs aligned to 32 bytes (and more than one sequence) run as ONE set of
+ * launches over all sequences: every (sequence, head[, segment]) is a thread block of the tensor-core kernels, which
+ * take each sequence's first token and length from a small table the call copies to the head of the workspace
+ * (a host-to-device copy on `stream` from pageable memory: such a call cannot be captured into a graph).  Other
+ * shapes enqueue one la_fwd / la_bwd per sequence on `stream`.  la_varlen_workspace_bytes covers both.
  */
 size_t la_varlen_workspace_bytes(int op, const la_shape* shape, const int* cu_seqlens_host, int num_seqs);
 la_status la_fwd_varlen(const la_shape* shape, const void* q, const void* k, const void* v, const float* lambda_host,

@@ -40,10 +40,19 @@ KernelTimer::~KernelTimer() {
 
 namespace {
 
+// A packed batch: sequences of different lengths one after the other in [total_tokens, H, D] tensors (DEVICE arrays
+// of first tokens and lengths, one entry per sequence); the shape that goes with it has B = sequences, N = longest.
+struct Packed {
+  const int* start;
+  const int* len;
+  int total_tokens;
+};
+
 struct Plan {
   int BH, seg_len, nseg;
   bool tensor;      // tensor-core kernels
   int precision;    // LA_SPLIT_* bits (tensor path)
+  Packed pk;        // start == NULL: dense batch
 };
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -75,6 +84,7 @@ bool tensor_path_available(const la_shape* s) {
 }
 
 la_status make_plan(const la_shape* s, Plan* p) {
+  p->pk = Packed{nullptr, nullptr, 0};
   p->BH = s->B * s->H;
   if (s->path == LA_PATH_TENSOR && !tensor_path_available(s)) return LA_ERR_UNSUPPORTED;
   p->tensor = (s->path == LA_PATH_TENSOR) || (s->path == LA_PATH_AUTO && tensor_path_available(s));
@@ -179,7 +189,10 @@ cudaError_t run_prepass(const la_shape* s, const Plan& p, const DecayTable& tab,
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
-  set_strides(s, s->N, &args);
+  args.seq_start = p.pk.start;
+  args.seq_len = p.pk.len;
+  args.total_tokens = p.pk.total_tokens;
+  set_strides(s, p.pk.start ? p.pk.total_tokens : s->N, &args);
   if (p.tensor) return launch_tc_prepass(args, tab, s->d, p.precision, st);
   return launch_simt_prepass(args, tab, s->d, s->e, (int)s->in_dtype, st);
 }
@@ -196,6 +209,7 @@ cudaError_t run_scan(const la_shape* s, const Plan& p, const DecayTable& tab, fl
   sa.N = s->N;
   sa.seg_len = p.seg_len;
   sa.nseg = p.nseg;
+  sa.seq_len = p.pk.len;
   sa.Da = s->d;  // d == e in every supported shape, so both orientations are square
   sa.Ec = s->e;
   sa.reverse = reverse;
@@ -217,7 +231,10 @@ OpArgs walk_args(const la_shape* s, const Plan& p, const void* a, const void* b,
   args.seg_len = p.seg_len;
   args.nseg = p.nseg;
   args.reverse = reverse;
-  set_strides(s, s->N, &args);
+  args.seq_start = p.pk.start;
+  args.seq_len = p.pk.len;
+  args.total_tokens = p.pk.total_tokens;
+  set_strides(s, p.pk.start ? p.pk.total_tokens : s->N, &args);
   return args;
 }
 
@@ -231,7 +248,11 @@ cudaError_t run_walk(const la_shape* s, const Plan& p, const DecayTable& tab, co
 
 la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
                    const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
-                   void* workspace, size_t workspace_bytes, void* stream);
+                   void* workspace, size_t workspace_bytes, void* stream, const Packed* pk = nullptr);
+la_status bwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* d_o,
+                   const float* lambda_host, void* dq, void* dk, void* dv, const float* kv_in,
+                   const float* grad_kv_out, float* grad_kv_in, const void* fwd_workspace, void* workspace,
+                   size_t workspace_bytes, void* stream, const Packed* pk);
 la_status decode_impl(const la_shape* shape, int T, const void* q, const void* k, const void* v,
                       const float* lambda_host, float* kv, void* o, void* stream);
 
@@ -305,7 +326,7 @@ namespace {
 // y = SRMSNorm(o) (.) u, fused into the walk where the kernel can, else by a row kernel behind it.
 la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* u,
                    const float* lambda_host, void* y, void* o, float* rstd, const float* kv_in, float* kv_out,
-                   void* workspace, size_t workspace_bytes, void* stream) {
+                   void* workspace, size_t workspace_bytes, void* stream, const Packed* pk) {
   la_status st = check_shape(shape, true);
   if (st != LA_OK) return st;
   if (!q || !k || !v || (!u && !o)) return LA_ERR_INVALID_ARG;
@@ -316,6 +337,7 @@ la_status fwd_impl(const la_shape* shape, const void* q, const void* k, const vo
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
   Plan p;
   if ((st = make_plan(shape, &p)) != LA_OK) return st;
+  if (pk) p.pk = *pk;
   const size_t one = state_set_bytes(shape, p);
   const size_t need = p.nseg > 1 ? 2 * one : 0;
   if (need > 0 && (!workspace || workspace_bytes < need)) return LA_ERR_WORKSPACE;
@@ -367,6 +389,18 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
                        const void* d_o, const float* lambda_host, void* dq, void* dk, void* dv,
                        const float* kv_in, const float* grad_kv_out, float* grad_kv_in,
                        const void* fwd_workspace, void* workspace, size_t workspace_bytes, void* stream) {
+  return bwd_impl(shape, q, k, v, d_o, lambda_host, dq, dk, dv, kv_in, grad_kv_out, grad_kv_in, fwd_workspace,
+                  workspace, workspace_bytes, stream, nullptr);
+}
+
+}  // extern "C"
+
+namespace la {
+namespace {
+la_status bwd_impl(const la_shape* shape, const void* q, const void* k, const void* v, const void* d_o,
+                   const float* lambda_host, void* dq, void* dk, void* dv, const float* kv_in,
+                   const float* grad_kv_out, float* grad_kv_in, const void* fwd_workspace, void* workspace,
+                   size_t workspace_bytes, void* stream, const Packed* pk) {
   la_status st = check_shape(shape, true);
   if (st != LA_OK) return st;
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return LA_ERR_INVALID_ARG;
@@ -378,6 +412,7 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
   if ((st = make_table(shape, lambda_host, &tab)) != LA_OK) return st;
   Plan p;
   if ((st = make_plan(shape, &p)) != LA_OK) return st;
+  if (pk) p.pk = *pk;
   const size_t one = state_set_bytes(shape, p);
   if (!workspace || workspace_bytes < 3 * one) return LA_ERR_WORKSPACE;
   if (fwd_workspace == workspace) return LA_ERR_INVALID_ARG;
@@ -424,6 +459,10 @@ la_status la_bwd_reuse(const la_shape* shape, const void* q, const void* k, cons
   }
   return LA_OK;
 }
+}  // namespace
+}  // namespace la
+
+extern "C" {
 
 la_status la_decode_step(const la_shape* shape, const void* q, const void* k, const void* v,
                          const float* lambda_host, float* kv, void* o, void* stream) {
@@ -706,6 +745,38 @@ la_status varlen_check(const la_shape* shape, const int* cu, int S, la_shape* su
   return LA_OK;
 }
 size_t esize(int dt) { return dt == LA_BF16 ? 2 : 4; }
+
+// The single-launch form: every sequence is a "batch" entry of its own length inside the packed tensors, and the
+// full-width tensor-core walk (with the state-only pre-pass and the scan where the longest sequence is cut into
+// segments) runs over all of them at once.  It exists for bf16 inputs at d = e = 128 with outputs aligned to 32
+// bytes; everything else runs one call per sequence.  `sp` is the shape that goes with it: B = sequences, N = longest.
+bool packed_shape(const la_shape* shape, const int* cu, int S, la_shape* sp) {
+  if (S < 2 || shape->d != 128 || shape->in_dtype != LA_BF16 || shape->path == LA_PATH_SIMT || !tc_supported())
+    return false;
+  int longest = 0;
+  for (int i = 0; i < S; ++i) longest = std::max(longest, cu[i + 1] - cu[i]);
+  *sp = *shape;
+  sp->B = S;
+  sp->N = longest;
+  return check_shape(sp, true) == LA_OK;
+}
+size_t packed_table_bytes(int S) { return ((size_t)2 * S * sizeof(int) + 255) / 256 * 256; }
+
+// Copies first tokens and lengths to the head of the workspace (stream-ordered) and describes them.
+la_status packed_upload(const int* cu, int S, int total, void* workspace, cudaStream_t cs, Packed* pk) {
+  std::vector<int> host(2 * (size_t)S);
+  for (int i = 0; i < S; ++i) {
+    host[i] = cu[i];
+    host[S + i] = cu[i + 1] - cu[i];
+  }
+  // pageable source: the runtime has taken its copy of the table by the time the call returns
+  if (cudaMemcpyAsync(workspace, host.data(), host.size() * sizeof(int), cudaMemcpyHostToDevice, cs) != cudaSuccess)
+    return LA_ERR_CUDA;
+  pk->start = static_cast<const int*>(workspace);
+  pk->len = pk->start + S;
+  pk->total_tokens = total;
+  return LA_OK;
+}
 }  // namespace
 
 size_t la_varlen_workspace_bytes(int op, const la_shape* shape, const int* cu_seqlens_host, int num_seqs) {
@@ -719,6 +790,11 @@ size_t la_varlen_workspace_bytes(int op, const la_shape* shape, const int* cu_se
     if (w == (size_t)-1) return (size_t)-1;
     if (w > most) most = w;
   }
+  la_shape sp;
+  if (packed_shape(shape, cu_seqlens_host, num_seqs, &sp)) {  // the single-launch form: its table and its state sets
+    const size_t w = la_workspace_bytes(op, &sp);
+    if (w != (size_t)-1 && packed_table_bytes(num_seqs) + w > most) most = packed_table_bytes(num_seqs) + w;
+  }
   return most;
 }
 
@@ -729,6 +805,17 @@ la_status la_fwd_varlen(const la_shape* shape, const void* q, const void* k, con
   la_status st = varlen_check(shape, cu_seqlens_host, num_seqs, &sub);
   if (st != LA_OK) return st;
   if (!q || !k || !v || !o) return LA_ERR_INVALID_ARG;
+  la_shape sp;
+  if (packed_shape(shape, cu_seqlens_host, num_seqs, &sp) && tc_walk_is_full(shape->d, o, nullptr)) {
+    const size_t tb = packed_table_bytes(num_seqs);
+    if (!workspace || workspace_bytes < tb || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return LA_ERR_WORKSPACE;
+    if ((st = check_device()) != LA_OK) return st;
+    Packed pk;
+    if ((st = packed_upload(cu_seqlens_host, num_seqs, shape->N, workspace, static_cast<cudaStream_t>(stream), &pk)) != LA_OK)
+      return st;
+    return fwd_impl(&sp, q, k, v, nullptr, lambda_host, nullptr, o, nullptr, kv_in, kv_out,
+                    static_cast<char*>(workspace) + tb, workspace_bytes - tb, stream, &pk);
+  }
   const size_t row_in = (size_t)shape->H * shape->d * esize(shape->in_dtype);
   const size_t row_out = (size_t)shape->H * shape->e * esize(shape->out_dtype);
   const size_t state = (size_t)shape->H * shape->d * shape->e;
@@ -752,6 +839,18 @@ la_status la_bwd_varlen(const la_shape* shape, const void* q, const void* k, con
   la_status st = varlen_check(shape, cu_seqlens_host, num_seqs, &sub);
   if (st != LA_OK) return st;
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return LA_ERR_INVALID_ARG;
+  la_shape sp;
+  if (packed_shape(shape, cu_seqlens_host, num_seqs, &sp) && tc_walk_is_full(shape->d, dq, dk) &&
+      tc_walk_is_full(shape->d, dv, nullptr)) {
+    const size_t tb = packed_table_bytes(num_seqs);
+    if (!workspace || workspace_bytes < tb || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return LA_ERR_WORKSPACE;
+    if ((st = check_device()) != LA_OK) return st;
+    Packed pk;
+    if ((st = packed_upload(cu_seqlens_host, num_seqs, shape->N, workspace, static_cast<cudaStream_t>(stream), &pk)) != LA_OK)
+      return st;
+    return bwd_impl(&sp, q, k, v, d_o, lambda_host, dq, dk, dv, kv_in, grad_kv_out, grad_kv_in, nullptr,
+                    static_cast<char*>(workspace) + tb, workspace_bytes - tb, stream, &pk);
+  }
   const size_t row_in = (size_t)shape->H * shape->d * esize(shape->in_dtype);
   const size_t row_out = (size_t)shape->H * shape->e * esize(shape->out_dtype);
   const size_t state = (size_t)shape->H * shape->d * shape->e;

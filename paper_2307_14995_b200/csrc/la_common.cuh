@@ -57,6 +57,15 @@ struct OpArgs {
   const void* u;      // [BH, N, Ec] gate, input dtype
   void* y;            // [BH, N, Ec] output dtype
   float* rstd;        // [BH, N] sqrt(Ec) / ||out row||_2, or NULL
+  // Packed batch of sequences of different lengths (tensor-core kernels at Da = Ec = 128 only; NULL elsewhere):
+  // the token tensors are [total_tokens, H, D] with the sequences one after the other, "batch" entry b is
+  // sequence b with seq_len[b] tokens starting at token seq_start[b] (DEVICE arrays of BH / H ints), N is the
+  // longest length (it fixes the segment grid; thread blocks of segments a sequence does not have return at once)
+  // and sB is unused.  Rows past a sequence's end belong to its neighbour, not to a zero-filled margin, so every
+  // bound below is the sequence's own length.
+  const int* seq_start;
+  const int* seq_len;
+  int total_tokens;
 };
 
 struct ScanArgs {
@@ -65,6 +74,7 @@ struct ScanArgs {
   const float* z_in;   // [BH, Da*Ec] (or [BH, Ec*Da] if z_in_transposed), or NULL = zeros
   int z_in_transposed;
   int BH, H, N, seg_len, nseg, Da, Ec, reverse;
+  const int* seq_len;  // packed batch: DEVICE array of BH / H lengths (N is then the longest), or NULL
 };
 
 // Chain of piece-local states into the state at one boundary (a cut of the sequence):
@@ -111,6 +121,8 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int
                            cudaStream_t stream);
 // Whether launch_tc_walk can fuse the epilogue described by args.u / args.y into the walk (d = 128, y and out
 // aligned to 32 bytes); otherwise the caller runs the walk and then launch_norm_gate_fwd.
+// True when launch_tc_walk / launch_tc_walk_pair take the full-width kernel for these outputs (D = 128, aligned to 32 bytes).
+bool tc_walk_is_full(int D, const void* out0, const void* out1);
 bool tc_can_fuse_gate(const OpArgs& args, int D);
 // Two walks of the same direction over the same tokens (same N, BH, segments) in one launch; the thread blocks of
 // the two are interleaved so that tiles both read come from HBM once.

@@ -300,8 +300,11 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs args, const De
   const int x0 = (blockIdx.y / tiles_y) * 32, y0 = (blockIdx.y % tiles_y) * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
   const double s2 = tab.s2[bh % args.H];
-  for (int p = threadIdx.x; p < args.nseg; p += 256) {
-    const int L = min(args.N, (p + 1) * args.seg_len) - p * args.seg_len;
+  // this (batch, head)'s own length and segment count (a packed batch has sequences of different lengths)
+  const int n_tok = args.seq_len ? args.seq_len[bh / args.H] : args.N;
+  const int nseg = (n_tok + args.seg_len - 1) / args.seg_len;
+  for (int p = threadIdx.x; p < nseg; p += 256) {
+    const int L = min(n_tok, (p + 1) * args.seg_len) - p * args.seg_len;
     gamma[p] = decay_pow_d(s2, (double)L);
   }
   float z[4];
@@ -314,17 +317,17 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs args, const De
   __syncthreads();
   // the local state of a segment is fetched one step ahead of its use: the chain over segments is
   // sequential, and this keeps one global-memory round trip out of every step
-  auto seg_of = [&](int ip) { return args.reverse ? (args.nseg - 1 - ip) : ip; };
+  auto seg_of = [&](int ip) { return args.reverse ? (nseg - 1 - ip) : ip; };
   float loc[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k)
-    loc[k] = (args.nseg > 1) ? args.buf[((size_t)bh * args.nseg + seg_of(0)) * DE + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] : 0.f;
-  for (int ip = 0; ip < args.nseg; ++ip) {
+    loc[k] = (nseg > 1) ? args.buf[((size_t)bh * args.nseg + seg_of(0)) * DE + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx] : 0.f;
+  for (int ip = 0; ip < nseg; ++ip) {
     const int p = seg_of(ip);
     const size_t off = ((size_t)bh * args.nseg + p) * DE;
-    const bool more = (ip + 1 < args.nseg);
+    const bool more = (ip + 1 < nseg);
     float nxt[4] = {0.f, 0.f, 0.f, 0.f};
-    if (ip + 2 < args.nseg) {
+    if (ip + 2 < nseg) {
       const size_t offn = ((size_t)bh * args.nseg + seg_of(ip + 1)) * DE;
 #pragma unroll
       for (int k = 0; k < 4; ++k) nxt[k] = args.buf[offn + (size_t)(x0 + ty + 8 * k) * Ec + y0 + tx];

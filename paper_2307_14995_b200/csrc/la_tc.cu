@@ -123,6 +123,8 @@ struct TcMaps {
 struct TcArgs {
   TcJob job[2];
   float* local_out;
+  const int* seq_start;  // packed batch (see OpArgs): DEVICE arrays, or NULL
+  const int* seq_len;
   int njobs;
   int BH, H, N, seg_len, nseg;
   int precision;
@@ -252,10 +254,16 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
   const int ehalf = (D == 128) ? (int)(bidx & 1) : 0;
   const int segid = (D == 128) ? (int)(bidx >> 1) : (int)bidx;
   const int bh = segid / args.nseg, seg = segid % args.nseg;
-  const int hh_ = bh % args.H, bb_ = bh / args.H;  // head and batch coordinates of the 4-D tensor maps
-  const size_t head_off = (size_t)bb_ * args.sB + (size_t)hh_ * args.sH;
+  const int hh_ = bh % args.H;  // head coordinate of the 4-D tensor maps
+  // Packed batch (state-only kernel; the walk of a packed batch is the full-width kernel's): entry bh / H is a
+  // sequence of its own length starting at token tok0 of one [tokens, H, D] tensor, the maps' batch coordinate is 0.
+  const int n_tok = args.seq_len ? args.seq_len[bh / args.H] : args.N;
+  const int tok0 = args.seq_start ? args.seq_start[bh / args.H] : 0;
+  const int bb_ = args.seq_start ? 0 : bh / args.H;
+  if (seg * args.seg_len >= n_tok) return;  // the grid covers the longest sequence; nothing has been set up yet
+  const size_t head_off = (size_t)bb_ * args.sB + (size_t)hh_ * args.sH + (size_t)tok0 * args.sT;
   const int seg_t0 = seg * args.seg_len;
-  const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
+  const int seg_t1 = min(n_tok, seg_t0 + args.seg_len);
   const float s2 = (float)tab.s2[bh % args.H];
   int nblk = (seg_t1 - seg_t0 + 127) >> 7;
   int it0 = 0;  // forward pre-pass: index of the first block that is walked
@@ -338,11 +346,11 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
         const int use = STATE_ONLY ? it / NLS : (it >> 1);  // how often this stage has been used before
         const uint32_t prev = (use - 1) & 1;                // parity of this stage's previous use
         const int blk = REV ? (nblk - 1 - it) : (it + it0);
-        const int t0 = seg_t0 + blk * 128;
+        const int t0 = tok0 + seg_t0 + blk * 128;  // token coordinate of the maps
         // State-only kernel: the tiles a few blocks ahead are pulled into L2 now, so that the loads proper are
         // L2 hits (measured: 0.276 -> 0.245 ms per launch; the same in the walk kernel made it slower).
         if (STATE_ONLY && it + NLS < nblk) {
-          const int tp = seg_t0 + (REV ? (nblk - 1 - NLS - it) : (it + NLS + it0)) * 128;
+          const int tp = tok0 + seg_t0 + (REV ? (nblk - 1 - NLS - it) : (it + NLS + it0)) * 128;
           tma_prefetch_4d(tm_b, 0, tp, hh_, bb_);
           if (D == 128) tma_prefetch_4d(tm_b, 64, tp, hh_, bb_);
           tma_prefetch_4d(tm_c, ehalf * 64, tp, hh_, bb_);
@@ -852,8 +860,10 @@ bool make_map(CUtensorMap* m, const void* ptr, const OpArgs& a, int D, bool f32 
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   const cuuint64_t esz = f32 ? 4 : 2;
-  const int B = a.BH / a.H;
-  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)a.N, (cuuint64_t)a.H, (cuuint64_t)B};
+  // packed batch: one [total_tokens, H, D] tensor, batch extent 1
+  const int B = a.seq_start ? 1 : a.BH / a.H;
+  const int tokens = a.seq_start ? a.total_tokens : a.N;
+  cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)tokens, (cuuint64_t)a.H, (cuuint64_t)B};
   cuuint64_t strides[3] = {(cuuint64_t)a.sT * esz, (cuuint64_t)a.sH * esz, (cuuint64_t)a.sB * esz};
   cuuint32_t box[4] = {(cuuint32_t)(128 / esz), 128, 1, 1};
   cuuint32_t es[4] = {1, 1, 1, 1};
@@ -899,6 +909,10 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
   ta.sT = args.sT; ta.sH = args.sH; ta.sB = args.sB;
+  ta.seq_start = args.seq_start;
+  ta.seq_len = args.seq_len;
+  if (args.seq_start && !tc_walk_is_full(D, args.out, second ? second->out : nullptr))
+    return cudaErrorInvalidValue;  // only the full-width kernel walks packed batches (the caller checks first)
   if (args.u) {
     // forward walk with the gate epilogue: only the full-width kernel has it (the caller asks tc_can_fuse_gate first)
     if (D != 128 || second || args.reverse || !tc_can_fuse_gate(args, D)) return cudaErrorInvalidValue;
@@ -948,6 +962,8 @@ cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int prec
   ta.BH = args.BH; ta.H = args.H; ta.N = args.N; ta.seg_len = args.seg_len; ta.nseg = args.nseg;
   ta.precision = precision;
   ta.sT = args.sT; ta.sH = args.sH; ta.sB = args.sB;
+  ta.seq_start = args.seq_start;
+  ta.seq_len = args.seq_len;
   return args.reverse ? launch_t<true, true, float, D, 1>(m, m, ta, tab, stream)
                       : launch_t<false, true, float, D, 1>(m, m, ta, tab, stream);
 }
@@ -963,6 +979,10 @@ cudaError_t launch_tc_walk(const OpArgs& args, const DecayTable& tab, int D, int
 }
 
 bool tc_full_width() { return true; }
+
+bool tc_walk_is_full(int D, const void* out0, const void* out1) {
+  return D == 128 && !((reinterpret_cast<uintptr_t>(out0) | reinterpret_cast<uintptr_t>(out1)) & 31u);
+}
 
 bool tc_can_fuse_gate(const OpArgs& args, int D) {
   if (D != 128 || !args.u || !args.y) return false;

@@ -85,10 +85,17 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
   if (NJOBS == 2 && jobid) job = args.job[1];
   const TcMaps& maps = (NJOBS == 2 && jobid) ? maps1 : maps0;
   const int bh = bidx / args.nseg, seg = bidx % args.nseg;
-  const int hh_ = bh % args.H, bb_ = bh / args.H;  // head and batch coordinates of the 4-D tensor maps
-  const size_t head_off = (size_t)bb_ * args.sB + (size_t)hh_ * args.sH;
+  const int hh_ = bh % args.H;  // head coordinate of the 4-D tensor maps
+  // Packed batch: "batch" entry bh / H is a sequence of its own length inside one [tokens, H, D] tensor; tok0 is its
+  // first token, and the maps' batch coordinate is 0.  Dense batch: tok0 = 0, every entry has N tokens.
+  const int n_tok = args.seq_len ? args.seq_len[bh / args.H] : args.N;
+  const int tok0 = args.seq_start ? args.seq_start[bh / args.H] : 0;
+  const int bb_ = args.seq_start ? 0 : bh / args.H;
+  const int nseg_own = (n_tok + args.seg_len - 1) / args.seg_len;
+  if (seg >= nseg_own) return;  // the grid covers the longest sequence; nothing has been set up yet
+  const size_t head_off = (size_t)bb_ * args.sB + (size_t)hh_ * args.sH + (size_t)tok0 * args.sT;
   const int seg_t0 = seg * args.seg_len;
-  const int seg_t1 = min(args.N, seg_t0 + args.seg_len);
+  const int seg_t1 = min(n_tok, seg_t0 + args.seg_len);
   const int nblk = (seg_t1 - seg_t0 + 127) >> 7;
   const float s2 = (float)tab.s2[bh % args.H];
   const bool split_p = (args.precision & 1) != 0;
@@ -128,7 +135,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
       // ------------------------------------ TMA producer ------------------------------------
       if (lane == 0) {
         for (int it = 0; it < nblk; ++it) {
-          const int t0 = seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;
+          const int t0 = tok0 + seg_t0 + (REV ? (nblk - 1 - it) : it) * 128;  // token coordinate of the maps
           // b is free once M3 of the previous block has read it (DZ_READY), a once M2 has (AB_FREE): each is
           // reloaded as soon as it falls free; both count towards the one barrier M1 of this block waits for
           if (it >= 1) TC_WAIT(F_DZ_READY, (it - 1) & 1, 3);
@@ -201,6 +208,10 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
     const int r = q * 32 + lane;       // score row
     const uint32_t colS = tmem + ((uint32_t)(q * 32) << 16) + FCOL_S;
     for (int it = 0; it < nblk; ++it) {
+      // Reverse walk, ragged block (the sequence's last tokens): the keys past the end lie inside the band.  In a
+      // dense batch they are the tensor maps' zero fill; in a packed batch they are the next sequence's tokens, so
+      // they are masked by index like the band itself.  (Forward walk: such keys are above the diagonal already.)
+      const int Cr_keys = REV ? min(128, seg_t1 - (seg_t0 + (nblk - 1 - it) * 128)) : 128;
       TC_WAIT_WARP(F_S_READY, it & 1, 17);
       tc_fence_after_sync();
 #pragma unroll 1
@@ -221,7 +232,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
 #pragma unroll
             for (int x = 0; x < 16; ++x) d[x] = ex2_approx(-s2 * (REV ? n0 + (float)x : n0 - (float)x));
             tmem_ld_wait();
-            if (REV ? (cc > q) : (cc < q)) {
+            if ((REV ? (cc > q) : (cc < q)) && Cr_keys == 128) {
               // 32x32 sub-tile wholly inside the causal band: nothing to mask
 #pragma unroll
               for (int x = 0; x < 16; ++x) d[x] = __uint_as_float(sreg[x]) * d[x];
@@ -231,7 +242,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
                 const int j = cc * 32 + hh * 16 + x;
                 const int n = REV ? (j - r) : (r - j);
                 // a select, not a multiply by zero: masked-out tokens can never leak
-                d[x] = (n >= 0) ? __uint_as_float(sreg[x]) * d[x] : 0.f;
+                d[x] = (n >= 0 && j < Cr_keys) ? __uint_as_float(sreg[x]) * d[x] : 0.f;
               }
             }
             split16(d, h8, l8);
@@ -296,7 +307,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
       const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(job.c) + head_off + (size_t)(t0 + frow) * args.sT + fch * 8;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        if (t0 + 32 * i + frow < args.N) raw[i] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(32 * i) * args.sT));
+        if (t0 + 32 * i + frow < n_tok) raw[i] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(32 * i) * args.sT));
         else raw[i] = make_uint4(0u, 0u, 0u, 0u);
       }
     };
@@ -362,7 +373,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
           WARP_ARRIVE(F_Z_READY);
         }
       }
-      const bool last_processed = REV ? (seg == 0) : (seg == args.nseg - 1);
+      const bool last_processed = REV ? (seg == 0) : (seg == nseg_own - 1);
       if (job.final_out && last_processed) {
         float* dst = job.final_out + (size_t)bh * (128 * 128) + (size_t)r * 128 + cg * 32;
 #pragma unroll

@@ -704,3 +704,44 @@ def test_packed_sequences_of_different_lengths(d):
         compare_all(got, ref, TOL_BF16)
     with pytest.raises(la.LaError):     # the description must cover the tensor exactly
         la.la_fwd_varlen(shape, qg, kg, vg, lam, o, cu[:-1] + [T - 1], None, None, ws_f)
+
+
+@pytest.mark.parametrize("seg_len,with_states", [(0, True), (256, True), (256, False)])
+def test_packed_batch_in_one_set_of_launches(seg_len, with_states):
+    """d = 128, bf16: all sequences of a packed batch run in the same launches (one walk launch when no sequence is
+    cut into segments; pre-pass, scan and walk otherwise), sequences end in the middle of 128-token blocks with the
+    next sequence's tokens right behind them, and every sequence is checked against the oracle on it alone."""
+    H, d = 2, 128
+    lens = [300, 1, 127, 128, 129, 1000, 64, 513]
+    cu = [0]
+    for n in lens:
+        cu.append(cu[-1] + n)
+    T, S = cu[-1], len(lens)
+    lam = torch.tensor([1.0, 0.9])
+    q, k, v, do = inputs.make_qkvdo(1, H, T, d, d, seed=95)
+    kv_in = inputs.make_state(S, H, d, d, seed=96) if with_states else None
+    gko = inputs.make_state(S, H, d, d, seed=97) if with_states else None
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(DEV)
+    qg, kg, vg, dog = tm(q), tm(k), tm(v), tm(do)
+    shape = la.make_shape(1, H, T, d, d, torch.bfloat16, torch.float32, seg_len, layout=la.LA_LAYOUT_BNHD)
+    o, dq, dk, dv = (torch.full((1, T, H, d), float("nan"), dtype=torch.float32, device=DEV) for _ in range(4))
+    kv_out, gin = (torch.empty((S, H, d, d), dtype=torch.float32, device=DEV) for _ in range(2))
+    ws_f = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_FWD, shape, cu), 256), dtype=torch.uint8, device=DEV)
+    ws_b = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_BWD, shape, cu), 256), dtype=torch.uint8, device=DEV)
+    kin = None if kv_in is None else kv_in.to(DEV)
+    gk = None if gko is None else gko.to(DEV)
+    l0 = la.launch_count()
+    la.la_fwd_varlen(shape, qg, kg, vg, lam, o, cu, kin, kv_out, ws_f)
+    assert la.launch_count() - l0 == (1 if seg_len == 0 else 3)
+    la.la_bwd_varlen(shape, qg, kg, vg, dog, lam, dq, dk, dv, cu, kin, gk, gin, ws_b)
+    torch.cuda.synchronize()
+    la.device_status()
+    back = lambda x, a, b: x[:, a:b].permute(0, 2, 1, 3)
+    for i in range(S):
+        a, b = cu[i], cu[i + 1]
+        ref = oracle_all(q[:, :, a:b], k[:, :, a:b], v[:, :, a:b], do[:, :, a:b], lam,
+                         None if kv_in is None else kv_in[i:i + 1].double().numpy(),
+                         None if gko is None else gko[i:i + 1].double().numpy())
+        got = (back(o, a, b), kv_out[i:i + 1], back(dq, a, b), back(dk, a, b), back(dv, a, b), gin[i:i + 1])
+        compare_all(got, ref, TOL_BF16)
+    assert not torch.isnan(o).any() and not torch.isnan(dq).any() and not torch.isnan(dk).any() and not torch.isnan(dv).any()
