@@ -1,6 +1,7 @@
 // C-ABI entry points (declared in include/la.h): argument validation, the
 // segment plan, workspace carving and the launch sequences.  Nothing here
 // computes attention; every step of the path runs in the kernels.
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 #include <vector>
@@ -45,6 +46,7 @@ namespace {
 struct Packed {
   const int* start;
   const int* len;
+  const int* order;  // sequence indices, longest first
   int total_tokens;
 };
 
@@ -84,7 +86,7 @@ bool tensor_path_available(const la_shape* s) {
 }
 
 la_status make_plan(const la_shape* s, Plan* p) {
-  p->pk = Packed{nullptr, nullptr, 0};
+  p->pk = Packed{nullptr, nullptr, nullptr, 0};
   p->BH = s->B * s->H;
   if (s->path == LA_PATH_TENSOR && !tensor_path_available(s)) return LA_ERR_UNSUPPORTED;
   p->tensor = (s->path == LA_PATH_TENSOR) || (s->path == LA_PATH_AUTO && tensor_path_available(s));
@@ -191,6 +193,7 @@ cudaError_t run_prepass(const la_shape* s, const Plan& p, const DecayTable& tab,
   args.reverse = reverse;
   args.seq_start = p.pk.start;
   args.seq_len = p.pk.len;
+  args.seq_order = p.pk.order;
   args.total_tokens = p.pk.total_tokens;
   set_strides(s, p.pk.start ? p.pk.total_tokens : s->N, &args);
   if (p.tensor) return launch_tc_prepass(args, tab, s->d, p.precision, st);
@@ -233,6 +236,7 @@ OpArgs walk_args(const la_shape* s, const Plan& p, const void* a, const void* b,
   args.reverse = reverse;
   args.seq_start = p.pk.start;
   args.seq_len = p.pk.len;
+  args.seq_order = p.pk.order;
   args.total_tokens = p.pk.total_tokens;
   set_strides(s, p.pk.start ? p.pk.total_tokens : s->N, &args);
   return args;
@@ -760,20 +764,24 @@ bool packed_shape(const la_shape* shape, const int* cu, int S, la_shape* sp) {
   sp->N = longest;
   return check_shape(sp, true) == LA_OK;
 }
-size_t packed_table_bytes(int S) { return ((size_t)2 * S * sizeof(int) + 255) / 256 * 256; }
+size_t packed_table_bytes(int S) { return ((size_t)3 * S * sizeof(int) + 255) / 256 * 256; }
 
 // Copies first tokens and lengths to the head of the workspace (stream-ordered) and describes them.
 la_status packed_upload(const int* cu, int S, int total, void* workspace, cudaStream_t cs, Packed* pk) {
-  std::vector<int> host(2 * (size_t)S);
+  std::vector<int> host(3 * (size_t)S);
   for (int i = 0; i < S; ++i) {
     host[i] = cu[i];
     host[S + i] = cu[i + 1] - cu[i];
+    host[2 * S + i] = i;
   }
+  // longest first (ties in the caller's order): the thread blocks of a launch are handed out in index order
+  std::stable_sort(host.begin() + 2 * S, host.end(), [&](int a, int b) { return host[S + a] > host[S + b]; });
   // pageable source: the runtime has taken its copy of the table by the time the call returns
   if (cudaMemcpyAsync(workspace, host.data(), host.size() * sizeof(int), cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return LA_ERR_CUDA;
   pk->start = static_cast<const int*>(workspace);
   pk->len = pk->start + S;
+  pk->order = pk->start + 2 * S;
   pk->total_tokens = total;
   return LA_OK;
 }

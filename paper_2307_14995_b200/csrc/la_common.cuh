@@ -65,6 +65,7 @@ struct OpArgs {
   // bound below is the sequence's own length.
   const int* seq_start;
   const int* seq_len;
+  const int* seq_order;  // the order in which thread blocks take the sequences (longest first), or NULL
   int total_tokens;
 };
 

@@ -125,6 +125,7 @@ struct TcArgs {
   float* local_out;
   const int* seq_start;  // packed batch (see OpArgs): DEVICE arrays, or NULL
   const int* seq_len;
+  const int* seq_order;
   int njobs;
   int BH, H, N, seg_len, nseg;
   int precision;
@@ -253,7 +254,9 @@ tc_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant__ TcMaps m
   const CUtensorMap* const tm_out = (NJOBS == 2 && jobid) ? &maps1.out : &maps0.out;
   const int ehalf = (D == 128) ? (int)(bidx & 1) : 0;
   const int segid = (D == 128) ? (int)(bidx >> 1) : (int)bidx;
-  const int bh = segid / args.nseg, seg = segid % args.nseg;
+  const int seg = segid % args.nseg;
+  int bh = segid / args.nseg;
+  if (args.seq_order) bh = args.seq_order[bh / args.H] * args.H + bh % args.H;  // packed batch: longest sequences first
   const int hh_ = bh % args.H;  // head coordinate of the 4-D tensor maps
   // Packed batch (state-only kernel; the walk of a packed batch is the full-width kernel's): entry bh / H is a
   // sequence of its own length starting at token tok0 of one [tokens, H, D] tensor, the maps' batch coordinate is 0.
@@ -911,6 +914,7 @@ cudaError_t launch_walk_d(const OpArgs& args, const OpArgs* second, const DecayT
   ta.sT = args.sT; ta.sH = args.sH; ta.sB = args.sB;
   ta.seq_start = args.seq_start;
   ta.seq_len = args.seq_len;
+  ta.seq_order = args.seq_order;
   if (args.seq_start && !tc_walk_is_full(D, args.out, second ? second->out : nullptr))
     return cudaErrorInvalidValue;  // only the full-width kernel walks packed batches (the caller checks first)
   if (args.u) {
@@ -964,6 +968,7 @@ cudaError_t launch_prepass_d(const OpArgs& args, const DecayTable& tab, int prec
   ta.sT = args.sT; ta.sH = args.sH; ta.sB = args.sB;
   ta.seq_start = args.seq_start;
   ta.seq_len = args.seq_len;
+  ta.seq_order = args.seq_order;
   return args.reverse ? launch_t<true, true, float, D, 1>(m, m, ta, tab, stream)
                       : launch_t<false, true, float, D, 1>(m, m, ta, tab, stream);
 }

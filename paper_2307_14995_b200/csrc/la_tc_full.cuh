@@ -84,7 +84,10 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
   TcJob job = args.job[0];
   if (NJOBS == 2 && jobid) job = args.job[1];
   const TcMaps& maps = (NJOBS == 2 && jobid) ? maps1 : maps0;
-  const int bh = bidx / args.nseg, seg = bidx % args.nseg;
+  const int seg = bidx % args.nseg;
+  int bh = bidx / args.nseg;
+  // packed batch: thread blocks take the sequences longest first, so that a long one is not what the launch ends on
+  if (args.seq_order) bh = args.seq_order[bh / args.H] * args.H + bh % args.H;
   const int hh_ = bh % args.H;  // head coordinate of the 4-D tensor maps
   // Packed batch: "batch" entry bh / H is a sequence of its own length inside one [tokens, H, D] tensor; tok0 is its
   // first token, and the maps' batch coordinate is 0.  Dense batch: tok0 = 0, every entry has N tokens.
