@@ -57,6 +57,30 @@ struct alignas(1024) FSmem {
   int abort;
 };
 
+// Clears, in the P tile a warp has just written to tensor memory (its 32 rows, 128 columns as 8 passes of 16:
+// words 0..7 of a pass hold the hi terms of column pairs (2x, 2x + 1), words 8..15 the lo terms), the columns from
+// `first` on.  Called once per thread block at most, by the whole warp; kept out of line so that the P group's
+// loop is compiled exactly as it is without it (a bound inside the loop cost the dense walk 1.5 %, this block
+// inlined behind it 0.4 %).
+__device__ __noinline__ void clear_keys_past_end(uint32_t colS, int first) {
+  tmem_st_wait();
+  for (int pass = first >> 4; pass < 8; ++pass) {
+    uint32_t w16[16];
+    tmem_ld_x16(colS + pass * 16, w16);
+    tmem_ld_wait();
+    uint32_t h8[8], l8[8];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+      const int j = pass * 16 + 2 * x;
+      const uint32_t keep = (j < first ? 0x0000ffffu : 0u) | (j + 1 < first ? 0xffff0000u : 0u);
+      h8[x] = w16[x] & keep;
+      l8[x] = w16[8 + x] & keep;
+    }
+    tmem_st_x8(colS + pass * 16, h8);
+    tmem_st_x8(colS + pass * 16 + 8, l8);
+  }
+}
+
 template <int N>
 __device__ __forceinline__ void reg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
@@ -211,10 +235,6 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
     const int r = q * 32 + lane;       // score row
     const uint32_t colS = tmem + ((uint32_t)(q * 32) << 16) + FCOL_S;
     for (int it = 0; it < nblk; ++it) {
-      // Reverse walk, ragged block (the sequence's last tokens): the keys past the end lie inside the band.  In a
-      // dense batch they are the tensor maps' zero fill; in a packed batch they are the next sequence's tokens, so
-      // they are masked by index like the band itself.  (Forward walk: such keys are above the diagonal already.)
-      const int Cr_keys = REV ? min(128, seg_t1 - (seg_t0 + (nblk - 1 - it) * 128)) : 128;
       TC_WAIT_WARP(F_S_READY, it & 1, 17);
       tc_fence_after_sync();
 #pragma unroll 1
@@ -235,7 +255,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
 #pragma unroll
             for (int x = 0; x < 16; ++x) d[x] = ex2_approx(-s2 * (REV ? n0 + (float)x : n0 - (float)x));
             tmem_ld_wait();
-            if ((REV ? (cc > q) : (cc < q)) && Cr_keys == 128) {
+            if (REV ? (cc > q) : (cc < q)) {
               // 32x32 sub-tile wholly inside the causal band: nothing to mask
 #pragma unroll
               for (int x = 0; x < 16; ++x) d[x] = __uint_as_float(sreg[x]) * d[x];
@@ -245,7 +265,7 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
                 const int j = cc * 32 + hh * 16 + x;
                 const int n = REV ? (j - r) : (r - j);
                 // a select, not a multiply by zero: masked-out tokens can never leak
-                d[x] = (n >= 0 && j < Cr_keys) ? __uint_as_float(sreg[x]) * d[x] : 0.f;
+                d[x] = (n >= 0) ? __uint_as_float(sreg[x]) * d[x] : 0.f;
               }
             }
             split16(d, h8, l8);
@@ -255,6 +275,10 @@ tc_walk_full_kernel(const __grid_constant__ TcMaps maps0, const __grid_constant_
           if (split_p) tmem_st_x8(colS + cc * 32 + hh * 16 + 8, l8);
         }
       }
+      // Reverse walk of a packed batch, the block that holds the sequence's last tokens: the keys past the end lie
+      // inside the band, and there they are the next sequence's tokens, not the zero fill a dense batch has.
+      if (REV && it == 0 && args.seq_start && seg_t1 - (seg_t0 + (nblk - 1) * 128) < 128)
+        clear_keys_past_end(colS, seg_t1 - (seg_t0 + (nblk - 1) * 128));
       tmem_st_wait();
       tc_fence_before_sync();
       WARP_ARRIVE(F_M4_OK);
