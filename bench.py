@@ -578,6 +578,32 @@ def run_ours(args):
         del od_, oo, odq, odk, odv, owf, owb, flush
 
     clocks = sampler.stop() if rank == 0 else None
+
+    # ---- the same step held for about two seconds (last GPU leg, so that it heats nothing that is timed after it):
+    # the headline loop above is a burst of a few tens of milliseconds from a GPU that was not under load just before;
+    # held for longer, the step runs into the board's power limit and the SM clock settles below its maximum
+    sustained = None
+    if train_steps and world == 1:
+        s_sampler = ClockSampler(local_rank)
+        n_hold = max(20, int(2000.0 / ms_step))
+        n_timed = n_hold // 2
+        for _ in range(n_hold - n_timed):
+            step()
+        s_sampler.start()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(n_timed):
+            step()
+        h1.record(stream)
+        torch.cuda.synchronize()
+        la.device_status()
+        s_clocks = s_sampler.stop()
+        s_ms = h0.elapsed_time(h1) / n_timed
+        sustained = {"what": "the same fwd+bwd step after %d untimed steps, mean of the next %d (about a second each)"
+                             % (n_hold - n_timed, n_timed),
+                     "ms_per_step": s_ms, "value": th * F / (s_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                     "step_roofline_frac": t_roof * 1e3 / s_ms, "clocks": s_clocks}
+
     cpu = cpu_baseline() if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
 
     if rank == 0:
@@ -602,7 +628,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / prof_steps for kname, (ms, _) in prof.items()},
             "kernel_launches_per_step": {kname: c / prof_steps for kname, (_, c) in prof.items()},
-            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe, "sequence_parallel": seqpar_leg, "varlen_prefill": varlen_leg,
+            "fwd_ms": split_ms.get("fwd"), "bwd_ms": split_ms.get("bwd"), "gated_forward": gated, "lrpe_d": lrpe, "sequence_parallel": seqpar_leg, "varlen_prefill": varlen_leg, "sustained": sustained,
             "roofline": {"scope": "ONE kernel, the dominant one; the whole-step figure the target is stated on is step_roofline",
                          "kernel": "full-width block walk (tc_walk_full_kernel), single-job launches (O and dQ)", "bound": "hbm",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
