@@ -745,3 +745,36 @@ def test_packed_batch_in_one_set_of_launches(seg_len, with_states):
         got = (back(o, a, b), kv_out[i:i + 1], back(dq, a, b), back(dk, a, b), back(dv, a, b), gin[i:i + 1])
         compare_all(got, ref, TOL_BF16)
     assert not torch.isnan(o).any() and not torch.isnan(dq).any() and not torch.isnan(dk).any() and not torch.isnan(dv).any()
+
+
+def test_packed_batch_bf16_outputs():
+    """The single-launch packed path with bf16 outputs (forward and backward), each sequence against the oracle."""
+    H, d = 2, 128
+    lens = [200, 77, 640]
+    cu = [0, 200, 277, 917]
+    T, S = cu[-1], len(lens)
+    lam = torch.tensor([0.99, 0.7])
+    q, k, v, do = inputs.make_qkvdo(1, H, T, d, d, seed=98)
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(DEV)
+    qg, kg, vg, dog = tm(q), tm(k), tm(v), tm(do)
+    shape = la.make_shape(1, H, T, d, d, torch.bfloat16, torch.bfloat16, 256, layout=la.LA_LAYOUT_BNHD)
+    o, dq, dk, dv = (torch.zeros((1, T, H, d), dtype=torch.bfloat16, device=DEV) for _ in range(4))
+    ws_f = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_FWD, shape, cu), 256), dtype=torch.uint8, device=DEV)
+    ws_b = torch.empty(max(la.varlen_workspace_bytes(la.LA_OP_BWD, shape, cu), 256), dtype=torch.uint8, device=DEV)
+    l0 = la.launch_count()
+    la.la_fwd_varlen(shape, qg, kg, vg, lam, o, cu, None, None, ws_f)
+    assert la.launch_count() - l0 == 3
+    la.la_bwd_varlen(shape, qg, kg, vg, dog, lam, dq, dk, dv, cu, None, None, None, ws_b)
+    torch.cuda.synchronize()
+    la.device_status()
+    back = lambda x, a, b: x[:, a:b].permute(0, 2, 1, 3).double().cpu().numpy()
+    lam64 = lam.double().numpy()
+    for i in range(S):
+        a, b = cu[i], cu[i + 1]
+        sl = lambda x: x[:, :, a:b]
+        ref_o = orc.fwd_rec(sl(q), sl(k), sl(v), lam64)
+        refs = (ref_o,) + tuple(orc.bwd_rec(sl(q), sl(k), sl(v), sl(do), lam64))
+        for got, ref, name in zip((o, dq, dk, dv), refs, ("o", "dq", "dk", "dv")):
+            g = back(got, a, b)
+            rms = np.sqrt(np.mean(ref * ref, axis=(2, 3), keepdims=True))
+            assert np.all(np.abs(g - ref) <= TOL_BF16 * rms + 2.0 ** -8 * np.abs(ref)), (name, i)
