@@ -155,19 +155,32 @@ __global__ void __launch_bounds__(256) lrpe_grad_kernel(const TIn* __restrict__ 
   }
 }
 
-// dtheta[h][i] = sum over the batch and the tiles of the two partial arrays, in a fixed order, in double.
-__global__ void lrpe_theta_reduce_kernel(const float* __restrict__ part_q, const float* __restrict__ part_k,
-                                         float* __restrict__ dtheta, int B, int H, int ntiles, int d) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= H * d) return;
-  const int h = idx / d, i = idx % d;
+// dtheta[h][i] = sum over the batch and the tiles of the two partial arrays, in double, in an order that depends on
+// the shape only (32 slices per feature: slice l adds the partials l, l + 32, ...; the slices are then added in
+// order through shared memory), so the result is reproducible bit for bit.  Eight consecutive features per block.
+__global__ void __launch_bounds__(256) lrpe_theta_reduce_kernel(const float* __restrict__ part_q,
+                                                                const float* __restrict__ part_k,
+                                                                float* __restrict__ dtheta, int B, int H, int ntiles, int d) {
+  const int slice = threadIdx.x >> 3, fi = threadIdx.x & 7;
+  const int idx = blockIdx.x * 8 + fi;  // feature index in [0, H*d)
+  __shared__ double red[32][8];
   double s = 0.0;
-  for (int b = 0; b < B; ++b)
-    for (int tl = 0; tl < ntiles; ++tl) {
+  if (idx < H * d) {
+    const int h = idx / d, i = idx % d;
+    const int n = B * ntiles;
+    for (int j = slice; j < n; j += 32) {
+      const int b = j / ntiles, tl = j % ntiles;
       const size_t at = ((size_t)(b * H + h) * ntiles + tl) * d + i;
       s += (double)part_q[at] + (double)part_k[at];
     }
-  dtheta[idx] = (float)s;
+  }
+  red[slice][fi] = s;
+  __syncthreads();
+  if (slice == 0 && idx < H * d) {
+    double t = 0.0;
+    for (int j = 0; j < 32; ++j) t += red[j][fi];
+    dtheta[idx] = (float)t;
+  }
 }
 
 unsigned grid_for(long threads_needed) {
@@ -370,8 +383,7 @@ la_status la_lrpe_bwd(const la_shape* shape, const void* q, const void* k, const
   {
     KernelTimer timer(K_LRPE, cs);
     const int n = shape->H * shape->d;
-    lrpe_theta_reduce_kernel<<<(n + 127) / 128, 128, 0, cs>>>(part_q, part_k, d_theta, shape->B, shape->H, c.ntiles,
-                                                             shape->d);
+    lrpe_theta_reduce_kernel<<<(n + 7) / 8, 256, 0, cs>>>(part_q, part_k, d_theta, shape->B, shape->H, c.ntiles, shape->d);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return LA_ERR_CUDA;
   }
