@@ -623,7 +623,7 @@ def run_ours(args):
                                      for kn, fv in flop_conventions(w.d).items()},
                        "bytes_per_token_head": bytes_per_token_head(w.d, ob, "step"),
                        "timing": "headline loop: profiling off, CUDA events on the launching stream; "
-                                 "kernel_ms_per_step and roofline come from a second, separately run profiled loop"},
+                                 "kernel_ms_per_step and roofline come from a second, separately run profiled loop; the board reaches its 1000 W power limit after about 40 ms of this step (15-18 steps from idle) and lowers the SM clock, so a run with more timed steps than that mixes both regimes: ms_per_step_median and ms_per_step_min show the full-clock steps, `sustained` the settled state"},
             "tokens_per_s": world * w.B * w.N / (ms_step * 1e-3),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "other_workloads": others,
             "kernel_ms_per_step": {kname: ms / prof_steps for kname, (ms, _) in prof.items()},
