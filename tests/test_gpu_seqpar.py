@@ -126,3 +126,25 @@ def test_single_rank_nccl_group_equals_the_plain_calls():
             assert torch.equal(a, b)
     finally:
         dist.destroy_process_group()
+
+
+def test_chunk_state_token_major_layout():
+    """la_chunk_state on [B,N,H,d] tensors gives the same states as on [B,H,N,d] ones, bit for bit."""
+    B, H, N, d = 2, 3, 600, 128
+    q, k, v, do = inputs.make_qkvdo(B, H, N, d, d, seed=36)
+    lam = torch.tensor([1.0, 0.95, 0.6])
+    out = {}
+    for name, layout in (("bhnd", la.LA_LAYOUT_BHND), ("bnhd", la.LA_LAYOUT_BNHD)):
+        tm = (lambda x: x.permute(0, 2, 1, 3).contiguous()) if layout == la.LA_LAYOUT_BNHD else (lambda x: x)
+        shape = la.make_shape(B, H, N, d, d, torch.bfloat16, torch.float32, 256, layout=layout)
+        ws = torch.empty(max(la.chunk_state_workspace_bytes(shape), 256), dtype=torch.uint8, device=DEV)
+        s_f = torch.empty((B, H, d, d), dtype=torch.float32, device=DEV)
+        s_r = torch.empty_like(s_f)
+        la.la_chunk_state(shape, 0, tm(k).to(DEV), tm(v).to(DEV), lam, s_f, ws)
+        la.la_chunk_state(shape, 1, tm(q).to(DEV), tm(do).to(DEV), lam, s_r, ws)
+        torch.cuda.synchronize()
+        out[name] = (s_f.clone(), s_r.clone())
+    la.device_status()
+    assert torch.equal(out["bhnd"][0], out["bnhd"][0]) and torch.equal(out["bhnd"][1], out["bnhd"][1])
+    _, kv = orc.fwd_rec(q, k, v, lam.double().numpy(), want_state=True)
+    assert_close(out["bnhd"][0], kv, TOL_BF16, "chunk state, token-major")
